@@ -1,0 +1,146 @@
+"""Pins for the oracle's DP active set and spMspV result (Sec. 2.2; Sec. 3.2; Sec. 4.2).
+
+Nothing here calls the CUDA library.
+"""
+import os
+
+import numpy as np
+import pytest
+
+from oracle import spdp_oracle as O
+from paper_2607_21985_b200 import workloads as WL
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _f16(a):
+    return np.asarray(a, dtype=np.float16)
+
+
+def test_active_rule_edge_vector():
+    thr = np.float16(0.5)
+    up = np.nextafter(thr, np.float16(np.inf))
+    dn = np.nextafter(thr, np.float16(0))
+    x = _f16([0.0, -0.0, thr, -thr, up, -up, dn, -dn, np.nan, np.inf, -np.inf, 6e-8, -6e-8, 65504, 1.0])
+    got = O.active_ref(x, O.DP_ABS_GT, float(thr))
+    #        0    -0     thr    -thr   up    -up   dn     -dn    nan   inf   -inf  sub    -sub   max   1
+    want = [False, False, False, False, True, True, False, False, True, True, True, False, False, True, True]
+    assert got.tolist() == want
+    # thr = 0 skips exactly the zeros; a negative thr keeps everything; NONE keeps everything
+    assert O.active_ref(x, O.DP_ABS_GT, 0.0).tolist() == [False, False] + [True] * 13
+    assert O.active_ref(x, O.DP_ABS_GT, -1.0).all() and O.active_ref(x, O.DP_NONE).all()
+    # explicit mask: bit j%32 of word j//32
+    m = np.zeros(40, bool)
+    m[[0, 5, 31, 32, 39]] = True
+    words = O.active_to_words(m)
+    assert words.tolist() == [(1 << 0) | (1 << 5) | (1 << 31), (1 << 0) | (1 << 7)]
+    assert np.array_equal(O.active_ref(np.zeros(40, np.float16), O.DP_MASK, mask_words=words), m)
+
+
+@pytest.mark.parametrize("skip", [0.0, 0.25, 0.4, 0.5, 0.9, 1.0])
+def test_threshold_recipe_hits_order_statistic(skip):
+    rng = np.random.Generator(np.random.PCG64(7))
+    x = rng.standard_normal(4096, dtype=np.float32).astype(np.float16)
+    rule, thr = WL.skip_threshold(x, skip)
+    a = O.active_ref(x, rule, thr)
+    assert abs((~a).sum() - round(skip * 4096)) <= 2          # ties at the cut can only add a few
+
+
+def test_sparsity_composition_paper_example():
+    """Sec. 3.2.2: independent masks overlap in sp*dp of the entries, total 1-(1-sp)(1-dp)."""
+    with open(os.path.join(GOLD, "sparsity_composition.txt")) as f:
+        rows = [l.split() for l in f if l.strip() and not l.startswith("#")]
+    sp, dp, overlap, total = map(float, rows[0])
+    assert abs(sp * dp - overlap) < 1e-12 and abs(1 - (1 - sp) * (1 - dp) - total) < 1e-12
+    M, K = 512, 2048
+    rw = np.random.Generator(np.random.PCG64(5))
+    G = WL.prune_global_magnitude(WL.normal_weights(rw, M, K), sp)
+    W = G.astype(np.float16)
+    x = rw.standard_normal(K, dtype=np.float32).astype(np.float16)
+    rule, thr = WL.skip_threshold(x, dp)
+    a = O.active_ref(x, rule, thr)
+    zero_w = ~O.is_nonzero(W)
+    both = (zero_w & ~a[None, :]).mean()
+    either = (zero_w | ~a[None, :]).mean()
+    assert abs(both - overlap) < 0.01 and abs(either - total) < 0.01
+
+
+def test_dense_gemv_special_case():
+    """0 % weight sparsity and no DP: the result is the library matrix-vector product."""
+    rng = np.random.Generator(np.random.PCG64(3))
+    W = (rng.standard_normal((300, 200), dtype=np.float32) * np.float32(0.02)).astype(np.float16)
+    x = rng.standard_normal(200, dtype=np.float32).astype(np.float16)
+    y, S = O.spmspv_ref(W, x, O.active_ref(x, O.DP_NONE))
+    ref = W.astype(np.float64) @ x.astype(np.float64)
+    assert np.allclose(y, ref, rtol=1e-13, atol=1e-15)
+    assert np.all(S >= np.abs(y) - 1e-12)
+
+
+def test_bruteforce_and_exact_integers():
+    rng = np.random.Generator(np.random.PCG64(9))
+    M, K = 70, 50
+    W = rng.integers(-8, 9, (M, K)).astype(np.float16)
+    W[rng.random((M, K)) < 0.5] = 0
+    x = rng.integers(-4, 5, K).astype(np.float16)
+    a = O.active_ref(x, O.DP_ABS_GT, 1.0)                      # skips |x| <= 1
+    y, S = O.spmspv_ref(W, x, a)
+    yb, Sb = O.spmspv_bruteforce(W, x, a)
+    assert np.array_equal(y, yb) and np.array_equal(S, Sb)     # integer sums are exact
+    # by hand on the integers
+    Wi, xi = W.astype(np.int64), x.astype(np.int64)
+    keep = np.abs(xi) > 1
+    assert np.array_equal(y, (Wi[:, keep] @ xi[keep]).astype(np.float64))
+    assert np.array_equal(S, (np.abs(Wi[:, keep]) @ np.abs(xi[keep])).astype(np.float64))
+
+
+def test_linearity_zeroed_x():
+    """Skipping a column equals multiplying by an x whose skipped entries are zero (finite W)."""
+    rng = np.random.Generator(np.random.PCG64(4))
+    W = (rng.standard_normal((128, 96), dtype=np.float32)).astype(np.float16)
+    W[rng.random(W.shape) < 0.6] = 0
+    x = rng.standard_normal(96, dtype=np.float32).astype(np.float16)
+    a = O.active_ref(x, O.DP_ABS_GT, 0.7)
+    y, _ = O.spmspv_ref(W, x, a)
+    xz = x.copy()
+    xz[~a] = 0
+    assert np.allclose(y, W.astype(np.float64) @ xz.astype(np.float64), rtol=1e-13, atol=1e-15)
+
+
+def test_inactive_columns_are_omitted_not_multiplied():
+    W = np.zeros((4, 3), np.float16)
+    W[0, 0] = np.inf
+    W[1, 1] = 2.0
+    x = _f16([0.0, 3.0, 1.0])
+    y, S = O.spmspv_ref(W, x, O.active_ref(x, O.DP_ABS_GT, 0.0))
+    assert y.tolist() == [0.0, 6.0, 0.0, 0.0] and S.tolist() == [0.0, 6.0, 0.0, 0.0]
+
+
+def test_permuted_identity_is_a_gather():
+    rng = np.random.Generator(np.random.PCG64(6))
+    n = 300
+    perm = rng.permutation(n)
+    W = np.zeros((n, n), np.float16)
+    W[np.arange(n), perm] = 1.0
+    x = rng.standard_normal(n, dtype=np.float32).astype(np.float16)
+    a = O.active_ref(x, O.DP_ABS_GT, 0.3)
+    y, _ = O.spmspv_ref(W, x, a)
+    want = np.where(a[perm], x[perm].astype(np.float64), 0.0)
+    assert np.array_equal(y, want)
+
+
+def test_all_columns_inactive_gives_zero():
+    W = np.ones((10, 8), np.float16)
+    x = np.full(8, 0.25, np.float16)
+    y, S = O.spmspv_ref(W, x, O.active_ref(x, O.DP_ABS_GT, 1.0))
+    assert not y.any() and not S.any()
+
+
+def test_result_from_packed_equals_result_from_dense():
+    """Decoding the packed arrays with the rule of Sec. 4.2.1 and multiplying gives the same y."""
+    W = WL.special_values_matrix(300, 40, 31)
+    W.view(np.uint16)[(W.view(np.uint16) & 0x7C00) == 0x7C00] = 0x3C00   # finite values only
+    x = np.random.Generator(np.random.PCG64(1)).standard_normal(40, dtype=np.float32).astype(np.float16)
+    a = O.active_ref(x, O.DP_ABS_GT, 0.5)
+    y, _ = O.spmspv_ref(W, x, a)
+    y2, _ = O.spmspv_ref(O.unpack_ref(O.pack_ref(W)), x, a)
+    assert np.array_equal(y, y2)

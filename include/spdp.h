@@ -1,0 +1,169 @@
+/* libspdp -- C ABI of the B200 (sm_100a) SPDP decode path.
+ *
+ * y = W_sp * (x masked by dynamic pruning): W_sp is an unstructured, statically pruned fp16
+ * matrix held in the Tiled-CBC format (Sec. 4.1 of the paper), x is one token's fp16
+ * activation vector, and columns whose activation fails the dynamic-pruning (DP) test are
+ * never fetched from device memory (Sec. 4.2).
+ *
+ * Conventions that hold for every call
+ *  - All tensor pointers named *_dev are CALLER-OWNED DEVICE memory on the device that was
+ *    current when the handle was created; pointers named *_host are host memory.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *  - Every call returns an spdp_status; nothing throws; out-parameters are written only on
+ *    SPDP_OK unless stated.  Host-detectable errors (null pointers, bad handle, unsupported
+ *    shape) are returned before any work is enqueued.
+ *  - A handle owns its packed arrays, its split-K workspace and a few staging buffers.  The
+ *    workspace is per handle, so at most ONE spdp_spmspv per handle may be in flight; calls on
+ *    one handle must be ordered (same stream, or events).  Different handles are independent.
+ *  - Format constants: column tile 256 x 1, GTile 256 x 16, four 64-bit bitmap words per column
+ *    tile (Sec. 4.1); 16-byte padding of every column's values (Sec. 4.2.3).
+ */
+#ifndef SPDP_H_
+#define SPDP_H_
+
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define SPDP_API __attribute__((visibility("default")))
+#else
+#define SPDP_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct spdp_matrix* spdp_handle;   /* opaque; created by pack/import, released by spdp_free */
+
+typedef enum {
+    SPDP_OK = 0,
+    SPDP_ERR_INVALID_ARG = -1,       /* null pointer, bad handle, bad enum, misaligned pointer */
+    SPDP_ERR_UNSUPPORTED_SHAPE = -2, /* tile shape other than 256 x 16, M or K < 1, ldw < K      */
+    SPDP_ERR_ALLOC = -3,             /* device or host allocation failed                        */
+    SPDP_ERR_CUDA = -4,              /* a CUDA runtime call failed (see spdp_last_cuda_error)    */
+    SPDP_ERR_OVERFLOW = -5,          /* Values would need 2^32 or more elements (TileOffset is 32-bit) */
+    SPDP_ERR_TIMEOUT = -6            /* a bounded device-side wait expired (device status word) */
+} spdp_status;
+
+/* Dynamic-pruning rule: which columns of W are fetched for this x (Sec. 2.2 "Dynamic Pruning",
+ * W_dp(x) = W (.) M(x); Sec. 4.2 step (3): a magnitude metric of the activation against a
+ * threshold calibrated offline, Sec. 5.1). */
+typedef enum {
+    SPDP_DP_NONE = 0,    /* every column is active                                              */
+    SPDP_DP_ABS_GT = 1,  /* column j active iff NOT(|x_j| <= thr), compared in fp32 on the exactly
+                            widened fp16 x_j: ties are skipped, thr = 0 skips exact zeros, thr < 0
+                            keeps everything, NaN and +-Inf activations are active             */
+    SPDP_DP_MASK = 2     /* explicit mask: bit (j % 32) of 32-bit word (j / 32) of mask_dev (Sec. 6:
+                            DP variants that materialise a mask use the same column interface)  */
+} spdp_dp_rule;
+
+typedef enum { SPDP_Y_F16 = 0, SPDP_Y_F32 = 1 } spdp_ydtype;
+
+/* Shape, sizes and device addresses of a packed matrix (all sizes in elements unless named bytes). */
+typedef struct {
+    int64_t M, K;              /* logical matrix shape                                          */
+    int64_t R, C, NGT;         /* row tiles ceil(M/256), GTile columns ceil(K/16), R*C          */
+    int64_t pad_elems;         /* every column's values are padded to a multiple of this (8 or 1) */
+    int64_t nnz;               /* stored nonzeros                                               */
+    int64_t values_len;        /* = TileOffset[NGT], padding included                           */
+    int64_t packed_bytes;      /* bytes of TileOffset + ColInfo + Bitmap + Values               */
+    int64_t workspace_bytes;   /* split-K scratch owned by the handle                           */
+    const void* tileoffset_dev;  /* uint32[NGT+1]  start of each GTile in Values (elements)      */
+    const void* colinfo_dev;     /* uint32[NGT*16] (column start inside its GTile) << 16 | nnz   */
+    const void* bitmap_dev;      /* uint64[NGT*16*4] bit b of word w = row 64*w+b of the column tile */
+    const void* values_dev;      /* fp16[values_len] nonzeros in tile-column order, zero padded  */
+    int32_t num_ctas;          /* CTAs one spdp_spmspv launches                                 */
+    int32_t device;            /* CUDA device ordinal the handle lives on                       */
+} spdp_info;
+
+/* Pack a dense, statically pruned matrix into Tiled-CBC (Sec. 4.1 "Storage Structure";
+ * padding rule of Sec. 4.2.3).
+ *   W_dev     fp16 [M][ldw] row-major, device; an element is "pruned" iff its value is +-0
+ *             (bits & 0x7FFF == 0); every other bit pattern, NaN/Inf/subnormals included, is
+ *             stored verbatim.
+ *   M, K      >= 1; sides that are not multiples of 256 / 16 are zero-extended logically.
+ *   ldw       leading dimension in elements, >= K.
+ *   tile_m, tile_k  must be 256 and 16 (the format's constants), else SPDP_ERR_UNSUPPORTED_SHAPE.
+ *   out       receives the handle.  The call allocates device memory, runs on `stream` and
+ *             synchronises it once (packing is an offline step).  W_dev is not retained.
+ * GTile (r, c) has linear index r*C + c; its 16 ColInfo words and 64 bitmap words are
+ * contiguous; Values holds, per GTile and per column, the column's nonzeros in row order
+ * followed by 0x0000 padding up to a multiple of 8 elements. */
+SPDP_API spdp_status spdp_pack_tiled_cbc(const void* W_dev, int64_t M, int64_t K, int64_t ldw,
+                                int tile_m, int tile_k, void* stream, spdp_handle* out);
+
+/* Same as spdp_pack_tiled_cbc with the padding unit chosen: pad_elems = 8 (the format) or 1 (no
+ * padding: the byte count then equals the storage formula of Sec. 4.1 exactly).  Handles packed
+ * with pad_elems = 1 can be inspected, exported and unpacked; spdp_spmspv rejects them with
+ * SPDP_ERR_UNSUPPORTED_SHAPE because its 16-byte loads need the padding. */
+SPDP_API spdp_status spdp_pack_tiled_cbc_ex(const void* W_dev, int64_t M, int64_t K, int64_t ldw,
+                                   int tile_m, int tile_k, int pad_elems, void* stream, spdp_handle* out);
+
+/* Build a handle from the four Tiled-CBC arrays in HOST memory (Sec. 4.1).  The arrays are
+ * validated on the host (monotone TileOffset, ColInfo offsets equal to the prefix sums of the
+ * padded counts, bitmap popcounts equal to the ColInfo counts); a mismatch returns
+ * SPDP_ERR_INVALID_ARG.  The data is copied; the host arrays are not retained. */
+SPDP_API spdp_status spdp_import_tiled_cbc(int64_t M, int64_t K, int pad_elems, const void* tileoffset_host,
+                                  const void* colinfo_host, const void* bitmap_host,
+                                  const void* values_host, int64_t values_len, spdp_handle* out);
+
+/* y = W_sp * x over the active columns only (Sec. 4.2, Alg. 1; fp32 accumulation).
+ *   x_dev     fp16 [K], device, 2-byte aligned.
+ *   rule/thr  the DP rule; thr is used by SPDP_DP_ABS_GT only.
+ *   mask_dev  uint32[ceil(K/32)], device; required for SPDP_DP_MASK, ignored otherwise.
+ *   y_dev     [M] of ydt (fp16 rounded to nearest even from the fp32 sum, or fp32), device.
+ *             Every one of the M entries is written, also when no column is active (zeros).
+ * Asynchronous on `stream`; allocates nothing and never synchronises.  Launches one kernel.
+ * The summation order is fixed for a given handle, so repeated calls give identical bits.
+ * Device-side problems (a bounded wait that expired) are recorded in the handle's device
+ * status word, readable with spdp_last_device_status. */
+SPDP_API spdp_status spdp_spmspv(spdp_handle h, const void* x_dev, spdp_dp_rule rule, float thr,
+                        const void* mask_dev, void* y_dev, spdp_ydtype ydt, void* stream);
+
+/* Same product with HOST vectors (Sec. 4.2): copies x_host (fp16 [K], ideally pinned) to a
+ * staging buffer of the handle, runs spdp_spmspv, copies y back into y_host ([M] of ydt) and
+ * synchronises `stream`.  mask_host is uint32[ceil(K/32)] or NULL. */
+SPDP_API spdp_status spdp_spmspv_host(spdp_handle h, const void* x_host, spdp_dp_rule rule, float thr,
+                             const void* mask_host, void* y_host, spdp_ydtype ydt, void* stream);
+
+/* Release the handle and everything it owns.  spdp_free(NULL) is SPDP_OK. */
+SPDP_API spdp_status spdp_free(spdp_handle h);
+
+/* ---- inspection surface (the format and the active set are checked bit for bit) ---- */
+
+SPDP_API spdp_status spdp_get_info(spdp_handle h, spdp_info* out);
+
+/* Copy the four arrays to HOST buffers sized as in spdp_info (any pointer may be NULL to skip
+ * it).  Synchronous. */
+SPDP_API spdp_status spdp_export(spdp_handle h, void* tileoffset_host, void* colinfo_host,
+                        void* bitmap_host, void* values_host);
+
+/* Decode the packed matrix back to dense fp16 [M][ldw] in device memory with the rule of
+ * Sec. 4.2.1 (bit clear -> +0, else Values[base + number of set bits before the position]).
+ * Asynchronous on `stream`. */
+SPDP_API spdp_status spdp_unpack(spdp_handle h, void* W_dev_out, int64_t ldw, void* stream);
+
+/* The active-column set spdp_spmspv would use for this x (Sec. 4.2 step (3)):
+ * bitmask_dev_out uint32[ceil(K/32)] (bit j%32 of word j/32, bits beyond K clear) and, if not
+ * NULL, count_dev_out int32[1], both device.  Asynchronous on `stream`. */
+SPDP_API spdp_status spdp_active_columns(spdp_handle h, const void* x_dev, spdp_dp_rule rule, float thr,
+                                const void* mask_dev, void* bitmask_dev_out, void* count_dev_out,
+                                void* stream);
+
+/* Read (and clear) the handle's device status word: 0, or an spdp_status recorded by a kernel.
+ * Synchronises the device. */
+SPDP_API spdp_status spdp_last_device_status(spdp_handle h, int* out);
+
+/* Tuning knob: number of CTAs spdp_spmspv launches (0 = default, one per SM).  Takes effect on
+ * the next call; re-derives the handle's split-K workspace layout (may reallocate it). */
+SPDP_API spdp_status spdp_set_num_ctas(spdp_handle h, int num_ctas);
+
+/* Text of the last CUDA runtime error seen by the library on this thread ("" if none). */
+SPDP_API const char* spdp_last_cuda_error(void);
+
+SPDP_API const char* spdp_status_string(spdp_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPDP_H_ */

@@ -1,0 +1,319 @@
+// C ABI of libspdp (declared in spdp.h): argument checks, handle life cycle, host-side layout
+// of the split-K work partition.  Every numerical step runs in the kernels of pack.cu and
+// spmspv.cu.
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "spdp_internal.h"
+
+namespace spdp {
+
+static thread_local char g_cuda_error[256] = "";
+
+void note_cuda_error(cudaError_t e, const char* what) {
+    std::snprintf(g_cuda_error, sizeof(g_cuda_error), "%s: %s (%s)", what, cudaGetErrorName(e),
+                  cudaGetErrorString(e));
+    cudaGetLastError();   // clear the sticky-free error state
+}
+
+namespace {
+
+void release(spdp_matrix* h) {
+    if (h == nullptr) return;
+    cudaFree(h->tileoffset);
+    cudaFree(h->colinfo);
+    cudaFree(h->bitmap);
+    cudaFree(h->values);
+    cudaFree(h->cta_begin);
+    cudaFree(h->row_first_cta);
+    cudaFree(h->row_nseg);
+    cudaFree(h->workspace);
+    cudaFree(h->row_counter);
+    cudaFree(h->status_word);
+    cudaFree(h->x_stage);
+    cudaFree(h->mask_stage);
+    cudaFree(h->y_stage);
+    h->magic = 0;
+    delete h;
+}
+
+spdp_status new_handle(int64_t M, int64_t K, int pad_elems, spdp_matrix** out) {
+    if (M < 1 || K < 1 || M > (int64_t(1) << 30) || K > (int64_t(1) << 30)) return SPDP_ERR_UNSUPPORTED_SHAPE;
+    if (pad_elems != 8 && pad_elems != 1) return SPDP_ERR_UNSUPPORTED_SHAPE;
+    spdp_matrix* h = new (std::nothrow) spdp_matrix();
+    if (h == nullptr) return SPDP_ERR_ALLOC;
+    std::memset(h, 0, sizeof(*h));
+    h->magic = kMagic;
+    h->M = M;
+    h->K = K;
+    h->R = (M + kTileM - 1) / kTileM;
+    h->C = (K + kTileK - 1) / kTileK;
+    h->NGT = h->R * h->C;
+    h->pad_elems = pad_elems;
+    if (h->NGT >= (int64_t(1) << 31) / kTileK) { delete h; return SPDP_ERR_UNSUPPORTED_SHAPE; }
+    cudaError_t e = cudaGetDevice(&h->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device);
+    if (e != cudaSuccess) { note_cuda_error(e, "device query"); delete h; return SPDP_ERR_CUDA; }
+    *out = h;
+    return SPDP_OK;
+}
+
+// Cuts the NGT GTiles into num_ctas equal contiguous ranges and derives, per row tile, which
+// CTAs feed it.  (Re)allocates the tables, the workspace and the counters.
+spdp_status build_partition(spdp_matrix* h, int num_ctas) {
+    const int64_t NGT = h->NGT, C = h->C, R = h->R;
+    int P = num_ctas > 0 ? num_ctas : h->sm_count;
+    if (P > NGT) P = static_cast<int>(NGT);
+    if (P < 1) P = 1;
+    std::vector<uint32_t> begin(P + 1);
+    for (int p = 0; p <= P; ++p) begin[p] = static_cast<uint32_t>((static_cast<__int128>(NGT) * p) / P);
+    std::vector<int32_t> first(R, -1), nseg(R, 0);
+    int max_segs = 1;
+    for (int p = 0; p < P; ++p) {
+        const int64_t r0 = begin[p] / C, r1 = (static_cast<int64_t>(begin[p + 1]) - 1) / C;
+        max_segs = max_segs > static_cast<int>(r1 - r0 + 1) ? max_segs : static_cast<int>(r1 - r0 + 1);
+        for (int64_t r = r0; r <= r1; ++r) {
+            if (first[r] < 0) first[r] = p;
+            ++nseg[r];
+        }
+    }
+    cudaFree(h->cta_begin);     h->cta_begin = nullptr;
+    cudaFree(h->row_first_cta); h->row_first_cta = nullptr;
+    cudaFree(h->row_nseg);      h->row_nseg = nullptr;
+    cudaFree(h->workspace);     h->workspace = nullptr;
+    cudaFree(h->row_counter);   h->row_counter = nullptr;
+    h->num_ctas = P;
+    h->max_segs = max_segs;
+    h->workspace_bytes = static_cast<int64_t>(P) * max_segs * kTileM * sizeof(float);
+    SPDP_CUDA_TRY(cudaMalloc(&h->cta_begin, (P + 1) * sizeof(uint32_t)));
+    SPDP_CUDA_TRY(cudaMalloc(&h->row_first_cta, R * sizeof(int32_t)));
+    SPDP_CUDA_TRY(cudaMalloc(&h->row_nseg, R * sizeof(int32_t)));
+    SPDP_CUDA_TRY(cudaMalloc(&h->workspace, h->workspace_bytes));
+    SPDP_CUDA_TRY(cudaMalloc(&h->row_counter, R * sizeof(unsigned)));
+    SPDP_CUDA_TRY(cudaMemcpy(h->cta_begin, begin.data(), (P + 1) * sizeof(uint32_t), cudaMemcpyHostToDevice));
+    SPDP_CUDA_TRY(cudaMemcpy(h->row_first_cta, first.data(), R * sizeof(int32_t), cudaMemcpyHostToDevice));
+    SPDP_CUDA_TRY(cudaMemcpy(h->row_nseg, nseg.data(), R * sizeof(int32_t), cudaMemcpyHostToDevice));
+    SPDP_CUDA_TRY(cudaMemset(h->workspace, 0, h->workspace_bytes));
+    SPDP_CUDA_TRY(cudaMemset(h->row_counter, 0, R * sizeof(unsigned)));
+    return SPDP_OK;
+}
+
+spdp_status finish_handle(spdp_matrix* h) {
+    spdp_status st = build_partition(h, 0);
+    if (st != SPDP_OK) return st;
+    SPDP_CUDA_TRY(cudaMalloc(&h->status_word, sizeof(int)));
+    SPDP_CUDA_TRY(cudaMemset(h->status_word, 0, sizeof(int)));
+    SPDP_CUDA_TRY(cudaMalloc(&h->x_stage, h->K * sizeof(__half)));
+    SPDP_CUDA_TRY(cudaMalloc(&h->mask_stage, ((h->K + 31) / 32) * sizeof(uint32_t)));
+    SPDP_CUDA_TRY(cudaMalloc(&h->y_stage, h->M * sizeof(float)));
+    return SPDP_OK;
+}
+
+bool rule_ok(int rule) { return rule == SPDP_DP_NONE || rule == SPDP_DP_ABS_GT || rule == SPDP_DP_MASK; }
+
+}  // namespace
+}  // namespace spdp
+
+using namespace spdp;
+
+extern "C" {
+
+spdp_status spdp_pack_tiled_cbc_ex(const void* W_dev, int64_t M, int64_t K, int64_t ldw, int tile_m,
+                                   int tile_k, int pad_elems, void* stream, spdp_handle* out) {
+    if (W_dev == nullptr || out == nullptr) return SPDP_ERR_INVALID_ARG;
+    if (tile_m != kTileM || tile_k != kTileK) return SPDP_ERR_UNSUPPORTED_SHAPE;
+    if (M < 1 || K < 1 || ldw < K) return SPDP_ERR_UNSUPPORTED_SHAPE;
+    if (reinterpret_cast<uintptr_t>(W_dev) & 1u) return SPDP_ERR_INVALID_ARG;
+    spdp_matrix* h = nullptr;
+    spdp_status st = new_handle(M, K, pad_elems, &h);
+    if (st != SPDP_OK) return st;
+    st = pack_device(h, static_cast<const __half*>(W_dev), ldw, static_cast<cudaStream_t>(stream));
+    if (st == SPDP_OK) st = finish_handle(h);
+    if (st != SPDP_OK) { release(h); return st; }
+    *out = h;
+    return SPDP_OK;
+}
+
+spdp_status spdp_pack_tiled_cbc(const void* W_dev, int64_t M, int64_t K, int64_t ldw, int tile_m,
+                                int tile_k, void* stream, spdp_handle* out) {
+    return spdp_pack_tiled_cbc_ex(W_dev, M, K, ldw, tile_m, tile_k, 8, stream, out);
+}
+
+spdp_status spdp_import_tiled_cbc(int64_t M, int64_t K, int pad_elems, const void* tileoffset_host,
+                                  const void* colinfo_host, const void* bitmap_host,
+                                  const void* values_host, int64_t values_len, spdp_handle* out) {
+    if (tileoffset_host == nullptr || colinfo_host == nullptr || bitmap_host == nullptr || out == nullptr)
+        return SPDP_ERR_INVALID_ARG;
+    if (values_len < 0 || (values_len > 0 && values_host == nullptr)) return SPDP_ERR_INVALID_ARG;
+    if (values_len >= (int64_t(1) << 32)) return SPDP_ERR_OVERFLOW;
+    spdp_matrix* h = nullptr;
+    spdp_status st = new_handle(M, K, pad_elems, &h);
+    if (st != SPDP_OK) return st;
+    const uint32_t* to = static_cast<const uint32_t*>(tileoffset_host);
+    const uint32_t* ci = static_cast<const uint32_t*>(colinfo_host);
+    const uint64_t* bm = static_cast<const uint64_t*>(bitmap_host);
+    // Structural validation of the arrays (Sec. 4.1): offsets are prefix sums of the padded counts.
+    int64_t nnz = 0;
+    bool ok = (to[0] == 0) && (static_cast<int64_t>(to[h->NGT]) == values_len);
+    for (int64_t g = 0; ok && g < h->NGT; ++g) {
+        int64_t off = 0;
+        for (int cc = 0; cc < kTileK; ++cc) {
+            const int64_t slot = g * kTileK + cc;
+            const int64_t n = ci[slot] & 0xFFFFu;
+            int64_t pc = 0;
+            for (int w = 0; w < kWordsPerCol; ++w) pc += __builtin_popcountll(bm[slot * kWordsPerCol + w]);
+            if (static_cast<int64_t>(ci[slot] >> 16) != off || pc != n) { ok = false; break; }
+            off += (n + pad_elems - 1) / pad_elems * pad_elems;
+            nnz += n;
+        }
+        if (ok && static_cast<int64_t>(to[g + 1]) - static_cast<int64_t>(to[g]) != off) ok = false;
+    }
+    if (!ok) { release(h); return SPDP_ERR_INVALID_ARG; }
+    h->nnz = nnz;
+    h->values_len = values_len;
+    const size_t vbytes = static_cast<size_t>(values_len) * sizeof(__half);
+    auto body = [&]() -> spdp_status {
+        SPDP_CUDA_TRY(cudaMalloc(&h->tileoffset, (h->NGT + 1) * sizeof(uint32_t)));
+        SPDP_CUDA_TRY(cudaMalloc(&h->colinfo, h->NGT * kTileK * sizeof(uint32_t)));
+        SPDP_CUDA_TRY(cudaMalloc(&h->bitmap, h->NGT * kTileK * kWordsPerCol * sizeof(uint64_t)));
+        SPDP_CUDA_TRY(cudaMalloc(&h->values, vbytes < 16 ? 16 : vbytes));
+        SPDP_CUDA_TRY(cudaMemset(h->values, 0, vbytes < 16 ? 16 : vbytes));
+        SPDP_CUDA_TRY(cudaMemcpy(h->tileoffset, to, (h->NGT + 1) * sizeof(uint32_t), cudaMemcpyHostToDevice));
+        SPDP_CUDA_TRY(cudaMemcpy(h->colinfo, ci, h->NGT * kTileK * sizeof(uint32_t), cudaMemcpyHostToDevice));
+        SPDP_CUDA_TRY(cudaMemcpy(h->bitmap, bm, h->NGT * kTileK * kWordsPerCol * sizeof(uint64_t),
+                                 cudaMemcpyHostToDevice));
+        if (vbytes) SPDP_CUDA_TRY(cudaMemcpy(h->values, values_host, vbytes, cudaMemcpyHostToDevice));
+        return finish_handle(h);
+    };
+    st = body();
+    if (st != SPDP_OK) { release(h); return st; }
+    *out = h;
+    return SPDP_OK;
+}
+
+spdp_status spdp_spmspv(spdp_handle h, const void* x_dev, spdp_dp_rule rule, float thr,
+                        const void* mask_dev, void* y_dev, spdp_ydtype ydt, void* stream) {
+    if (!valid(h) || x_dev == nullptr || y_dev == nullptr) return SPDP_ERR_INVALID_ARG;
+    if (!rule_ok(rule) || (ydt != SPDP_Y_F16 && ydt != SPDP_Y_F32)) return SPDP_ERR_INVALID_ARG;
+    if (rule == SPDP_DP_MASK && mask_dev == nullptr) return SPDP_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(x_dev) & 1u) ||
+        (reinterpret_cast<uintptr_t>(y_dev) & (ydt == SPDP_Y_F32 ? 3u : 1u)) ||
+        (reinterpret_cast<uintptr_t>(mask_dev) & 3u))
+        return SPDP_ERR_INVALID_ARG;
+    if (h->pad_elems != 8) return SPDP_ERR_UNSUPPORTED_SHAPE;
+    return launch_spmspv(h, static_cast<const __half*>(x_dev), rule, thr,
+                         static_cast<const uint32_t*>(mask_dev), y_dev, ydt, static_cast<cudaStream_t>(stream));
+}
+
+spdp_status spdp_spmspv_host(spdp_handle h, const void* x_host, spdp_dp_rule rule, float thr,
+                             const void* mask_host, void* y_host, spdp_ydtype ydt, void* stream) {
+    if (!valid(h) || x_host == nullptr || y_host == nullptr) return SPDP_ERR_INVALID_ARG;
+    if (!rule_ok(rule) || (ydt != SPDP_Y_F16 && ydt != SPDP_Y_F32)) return SPDP_ERR_INVALID_ARG;
+    if (rule == SPDP_DP_MASK && mask_host == nullptr) return SPDP_ERR_INVALID_ARG;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    SPDP_CUDA_TRY(cudaMemcpyAsync(h->x_stage, x_host, h->K * sizeof(__half), cudaMemcpyHostToDevice, s));
+    if (rule == SPDP_DP_MASK)
+        SPDP_CUDA_TRY(cudaMemcpyAsync(h->mask_stage, mask_host, ((h->K + 31) / 32) * sizeof(uint32_t),
+                                      cudaMemcpyHostToDevice, s));
+    spdp_status st = spdp_spmspv(h, h->x_stage, rule, thr, rule == SPDP_DP_MASK ? h->mask_stage : nullptr,
+                                 h->y_stage, ydt, stream);
+    if (st != SPDP_OK) return st;
+    const size_t ybytes = static_cast<size_t>(h->M) * (ydt == SPDP_Y_F32 ? sizeof(float) : sizeof(__half));
+    SPDP_CUDA_TRY(cudaMemcpyAsync(y_host, h->y_stage, ybytes, cudaMemcpyDeviceToHost, s));
+    SPDP_CUDA_TRY(cudaStreamSynchronize(s));
+    return SPDP_OK;
+}
+
+spdp_status spdp_free(spdp_handle h) {
+    if (h == nullptr) return SPDP_OK;
+    if (!valid(h)) return SPDP_ERR_INVALID_ARG;
+    release(h);
+    return SPDP_OK;
+}
+
+spdp_status spdp_get_info(spdp_handle h, spdp_info* out) {
+    if (!valid(h) || out == nullptr) return SPDP_ERR_INVALID_ARG;
+    spdp_info i;
+    std::memset(&i, 0, sizeof(i));
+    i.M = h->M; i.K = h->K; i.R = h->R; i.C = h->C; i.NGT = h->NGT;
+    i.pad_elems = h->pad_elems;
+    i.nnz = h->nnz;
+    i.values_len = h->values_len;
+    i.packed_bytes = (h->NGT + 1) * 4 + h->NGT * kTileK * 4 + h->NGT * kTileK * kWordsPerCol * 8 + h->values_len * 2;
+    i.workspace_bytes = h->workspace_bytes;
+    i.tileoffset_dev = h->tileoffset;
+    i.colinfo_dev = h->colinfo;
+    i.bitmap_dev = h->bitmap;
+    i.values_dev = h->values;
+    i.num_ctas = h->num_ctas;
+    i.device = h->device;
+    *out = i;
+    return SPDP_OK;
+}
+
+spdp_status spdp_export(spdp_handle h, void* tileoffset_host, void* colinfo_host, void* bitmap_host,
+                        void* values_host) {
+    if (!valid(h)) return SPDP_ERR_INVALID_ARG;
+    SPDP_CUDA_TRY(cudaDeviceSynchronize());
+    if (tileoffset_host)
+        SPDP_CUDA_TRY(cudaMemcpy(tileoffset_host, h->tileoffset, (h->NGT + 1) * sizeof(uint32_t), cudaMemcpyDeviceToHost));
+    if (colinfo_host)
+        SPDP_CUDA_TRY(cudaMemcpy(colinfo_host, h->colinfo, h->NGT * kTileK * sizeof(uint32_t), cudaMemcpyDeviceToHost));
+    if (bitmap_host)
+        SPDP_CUDA_TRY(cudaMemcpy(bitmap_host, h->bitmap, h->NGT * kTileK * kWordsPerCol * sizeof(uint64_t),
+                                 cudaMemcpyDeviceToHost));
+    if (values_host && h->values_len > 0)
+        SPDP_CUDA_TRY(cudaMemcpy(values_host, h->values, h->values_len * sizeof(__half), cudaMemcpyDeviceToHost));
+    return SPDP_OK;
+}
+
+spdp_status spdp_unpack(spdp_handle h, void* W_dev_out, int64_t ldw, void* stream) {
+    if (!valid(h) || W_dev_out == nullptr) return SPDP_ERR_INVALID_ARG;
+    if (ldw < h->K) return SPDP_ERR_UNSUPPORTED_SHAPE;
+    return unpack_device(h, static_cast<__half*>(W_dev_out), ldw, static_cast<cudaStream_t>(stream));
+}
+
+spdp_status spdp_active_columns(spdp_handle h, const void* x_dev, spdp_dp_rule rule, float thr,
+                                const void* mask_dev, void* bitmask_dev_out, void* count_dev_out,
+                                void* stream) {
+    if (!valid(h) || x_dev == nullptr || bitmask_dev_out == nullptr) return SPDP_ERR_INVALID_ARG;
+    if (!rule_ok(rule) || (rule == SPDP_DP_MASK && mask_dev == nullptr)) return SPDP_ERR_INVALID_ARG;
+    return launch_active_columns(h, static_cast<const __half*>(x_dev), rule, thr,
+                                 static_cast<const uint32_t*>(mask_dev), static_cast<uint32_t*>(bitmask_dev_out),
+                                 static_cast<int*>(count_dev_out), static_cast<cudaStream_t>(stream));
+}
+
+spdp_status spdp_last_device_status(spdp_handle h, int* out) {
+    if (!valid(h) || out == nullptr) return SPDP_ERR_INVALID_ARG;
+    int v = 0;
+    SPDP_CUDA_TRY(cudaDeviceSynchronize());
+    SPDP_CUDA_TRY(cudaMemcpy(&v, h->status_word, sizeof(int), cudaMemcpyDeviceToHost));
+    SPDP_CUDA_TRY(cudaMemset(h->status_word, 0, sizeof(int)));
+    *out = v;
+    return SPDP_OK;
+}
+
+spdp_status spdp_set_num_ctas(spdp_handle h, int num_ctas) {
+    if (!valid(h) || num_ctas < 0) return SPDP_ERR_INVALID_ARG;
+    SPDP_CUDA_TRY(cudaDeviceSynchronize());
+    return build_partition(h, num_ctas);
+}
+
+const char* spdp_last_cuda_error(void) { return g_cuda_error; }
+
+const char* spdp_status_string(spdp_status s) {
+    switch (s) {
+        case SPDP_OK: return "SPDP_OK";
+        case SPDP_ERR_INVALID_ARG: return "SPDP_ERR_INVALID_ARG";
+        case SPDP_ERR_UNSUPPORTED_SHAPE: return "SPDP_ERR_UNSUPPORTED_SHAPE";
+        case SPDP_ERR_ALLOC: return "SPDP_ERR_ALLOC";
+        case SPDP_ERR_CUDA: return "SPDP_ERR_CUDA";
+        case SPDP_ERR_OVERFLOW: return "SPDP_ERR_OVERFLOW";
+        case SPDP_ERR_TIMEOUT: return "SPDP_ERR_TIMEOUT";
+    }
+    return "SPDP_ERR_UNKNOWN";
+}
+
+}  // extern "C"

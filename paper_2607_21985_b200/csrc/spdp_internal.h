@@ -1,0 +1,78 @@
+// Internal declarations shared by the translation units of libspdp (not part of the ABI).
+#pragma once
+
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "spdp.h"
+
+namespace spdp {
+
+constexpr int kTileM = 256;        // rows per column tile (Sec. 4.1)
+constexpr int kTileK = 16;         // column tiles per GTile (Sec. 4.2.3)
+constexpr int kWordsPerCol = 4;    // 64-bit bitmap words per column tile (Sec. 4.1)
+constexpr uint64_t kMagic = 0x5350445042323030ull;   // "SPDPB200"
+
+}  // namespace spdp
+
+// Host-side state behind an spdp_handle.
+struct spdp_matrix {
+    uint64_t magic;
+    int device;
+    int sm_count;
+    int64_t M, K, R, C, NGT;
+    int pad_elems;
+    int64_t nnz;
+    int64_t values_len;
+
+    // Tiled-CBC arrays (device)
+    uint32_t* tileoffset;   // [NGT+1]
+    uint32_t* colinfo;      // [NGT*16]
+    uint64_t* bitmap;       // [NGT*16*4]
+    __half* values;         // [values_len] (at least 16 bytes are allocated)
+
+    // Work partition of one spmspv launch: CTA p owns GTiles [cta_begin[p], cta_begin[p+1]).
+    int num_ctas;           // P
+    int max_segs;           // most row tiles one CTA's range touches
+    uint32_t* cta_begin;    // device [P+1]
+    int32_t* row_first_cta; // device [R]: first CTA whose range touches row tile r
+    int32_t* row_nseg;      // device [R]: number of CTAs whose range touches row tile r
+    float* workspace;       // device [P*max_segs*256] split-K partial sums
+    unsigned* row_counter;  // device [R] arrivals per row tile (self-resetting)
+    int* status_word;       // device [1]
+    int64_t workspace_bytes;
+
+    // Staging for the host-vector entry point
+    __half* x_stage;        // device [K]
+    uint32_t* mask_stage;   // device [ceil(K/32)]
+    void* y_stage;          // device [M] fp32-sized
+};
+
+namespace spdp {
+
+// Records the message of a failed CUDA call for spdp_last_cuda_error().
+void note_cuda_error(cudaError_t e, const char* what);
+
+#define SPDP_CUDA_TRY(expr)                                   \
+    do {                                                      \
+        cudaError_t e__ = (expr);                             \
+        if (e__ != cudaSuccess) {                             \
+            ::spdp::note_cuda_error(e__, #expr);              \
+            return (e__ == cudaErrorMemoryAllocation) ? SPDP_ERR_ALLOC : SPDP_ERR_CUDA; \
+        }                                                     \
+    } while (0)
+
+inline bool valid(const spdp_matrix* h) { return h != nullptr && h->magic == kMagic; }
+
+// pack.cu
+spdp_status pack_device(spdp_matrix* h, const __half* W, int64_t ldw, cudaStream_t s);
+spdp_status unpack_device(const spdp_matrix* h, __half* W, int64_t ldw, cudaStream_t s);
+
+// spmspv.cu
+spdp_status launch_spmspv(const spdp_matrix* h, const __half* x, int rule, float thr,
+                          const uint32_t* mask, void* y, int ydt, cudaStream_t s);
+spdp_status launch_active_columns(const spdp_matrix* h, const __half* x, int rule, float thr,
+                                  const uint32_t* mask, uint32_t* bits, int* count, cudaStream_t s);
+
+}  // namespace spdp

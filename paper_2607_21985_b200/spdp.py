@@ -1,0 +1,220 @@
+"""ctypes binding of libspdp (include/spdp.h): same entry points, argument marshalling only.
+
+Tensors are torch CUDA tensors (their data_ptr() is handed to the library); the stream is
+torch's current stream unless given.  There is no fallback: if libspdp.so is missing the
+first call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libspdp.so")
+
+SPDP_OK = 0
+SPDP_ERR_INVALID_ARG = -1
+SPDP_ERR_UNSUPPORTED_SHAPE = -2
+SPDP_ERR_ALLOC = -3
+SPDP_ERR_CUDA = -4
+SPDP_ERR_OVERFLOW = -5
+SPDP_ERR_TIMEOUT = -6
+
+SPDP_DP_NONE, SPDP_DP_ABS_GT, SPDP_DP_MASK = 0, 1, 2
+SPDP_Y_F16, SPDP_Y_F32 = 0, 1
+
+EXPORTS = (
+    "spdp_pack_tiled_cbc", "spdp_pack_tiled_cbc_ex", "spdp_import_tiled_cbc", "spdp_spmspv",
+    "spdp_spmspv_host", "spdp_free", "spdp_get_info", "spdp_export", "spdp_unpack",
+    "spdp_active_columns", "spdp_last_device_status", "spdp_set_num_ctas", "spdp_last_cuda_error",
+    "spdp_status_string",
+)
+
+
+class spdp_info(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int64) for n in ("M", "K", "R", "C", "NGT", "pad_elems", "nnz", "values_len",
+                                              "packed_bytes", "workspace_bytes")] + \
+               [(n, ctypes.c_void_p) for n in ("tileoffset_dev", "colinfo_dev", "bitmap_dev", "values_dev")] + \
+               [("num_ctas", ctypes.c_int32), ("device", ctypes.c_int32)]
+
+
+class SpdpError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = lib().spdp_status_string(status).decode()
+        detail = lib().spdp_last_cuda_error().decode()
+        super().__init__(f"{where}: {msg}" + (f" [{detail}]" if detail and status in (-3, -4) else ""))
+
+
+_lib = None
+
+
+def lib():
+    """Loads libspdp.so (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2607_21985_b200.build` "
+                               "(there is no CPU fallback)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i64, ci, cf = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_float
+        L.spdp_pack_tiled_cbc.argtypes = [vp, i64, i64, i64, ci, ci, vp, ctypes.POINTER(vp)]
+        L.spdp_pack_tiled_cbc_ex.argtypes = [vp, i64, i64, i64, ci, ci, ci, vp, ctypes.POINTER(vp)]
+        L.spdp_import_tiled_cbc.argtypes = [i64, i64, ci, vp, vp, vp, vp, i64, ctypes.POINTER(vp)]
+        L.spdp_spmspv.argtypes = [vp, vp, ci, cf, vp, vp, ci, vp]
+        L.spdp_spmspv_host.argtypes = [vp, vp, ci, cf, vp, vp, ci, vp]
+        L.spdp_free.argtypes = [vp]
+        L.spdp_get_info.argtypes = [vp, ctypes.POINTER(spdp_info)]
+        L.spdp_export.argtypes = [vp, vp, vp, vp, vp]
+        L.spdp_unpack.argtypes = [vp, vp, i64, vp]
+        L.spdp_active_columns.argtypes = [vp, vp, ci, cf, vp, vp, vp, vp]
+        L.spdp_last_device_status.argtypes = [vp, ctypes.POINTER(ci)]
+        L.spdp_set_num_ctas.argtypes = [vp, ci]
+        for name in EXPORTS:
+            getattr(L, name).restype = ci
+        L.spdp_last_cuda_error.restype = ctypes.c_char_p
+        L.spdp_last_cuda_error.argtypes = []
+        L.spdp_status_string.restype = ctypes.c_char_p
+        L.spdp_status_string.argtypes = [ci]
+        _lib = L
+    return _lib
+
+
+def _check(st: int, where: str):
+    if st != SPDP_OK:
+        raise SpdpError(st, where)
+
+
+def _stream(stream):
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    return getattr(stream, "cuda_stream", stream)
+
+
+def _dev_ptr(t, name, allow_none=False):
+    if t is None:
+        if allow_none:
+            return None
+        raise ValueError(f"{name} is required")
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError(f"{name} must be a contiguous CUDA tensor")
+    return t.data_ptr()
+
+
+def _host_ptr(a, name, allow_none=False):
+    if a is None:
+        if allow_none:
+            return None
+        raise ValueError(f"{name} is required")
+    if isinstance(a, np.ndarray):
+        if not a.flags["C_CONTIGUOUS"]:
+            raise ValueError(f"{name} must be C-contiguous")
+        return a.ctypes.data
+    if a.is_cuda or not a.is_contiguous():       # torch CPU tensor (e.g. pinned)
+        raise ValueError(f"{name} must be a contiguous host tensor")
+    return a.data_ptr()
+
+
+# ---- the entry points, named as in spdp.h --------------------------------------------------
+def spdp_pack_tiled_cbc(W, tile_m: int = 256, tile_k: int = 16, stream=None, pad_elems: int | None = None) -> int:
+    """W: fp16 CUDA tensor [M, K] (row stride = ldw, unit column stride).  Returns the handle."""
+    import torch
+    if W.dtype != torch.float16 or W.dim() != 2 or not W.is_cuda or W.stride(1) != 1:
+        raise ValueError("W must be a 2-D fp16 CUDA tensor with unit column stride")
+    M, K = W.shape
+    h = ctypes.c_void_p()
+    if pad_elems is None:
+        st = lib().spdp_pack_tiled_cbc(W.data_ptr(), M, K, W.stride(0), tile_m, tile_k, _stream(stream), ctypes.byref(h))
+    else:
+        st = lib().spdp_pack_tiled_cbc_ex(W.data_ptr(), M, K, W.stride(0), tile_m, tile_k, pad_elems,
+                                          _stream(stream), ctypes.byref(h))
+    _check(st, "spdp_pack_tiled_cbc")
+    return h.value
+
+
+def spdp_import_tiled_cbc(M: int, K: int, tileoffset, colinfo, bitmap, values, pad_elems: int = 8) -> int:
+    """Host arrays (NumPy: uint32, uint32, uint64, uint16/float16) -> handle."""
+    to = np.ascontiguousarray(tileoffset, dtype=np.uint32)
+    ci = np.ascontiguousarray(colinfo, dtype=np.uint32)
+    bm = np.ascontiguousarray(bitmap, dtype=np.uint64)
+    va = np.ascontiguousarray(values)
+    if va.dtype == np.float16:
+        va = va.view(np.uint16)
+    if va.dtype != np.uint16:
+        raise ValueError("values must be uint16 bit patterns or float16")
+    h = ctypes.c_void_p()
+    st = lib().spdp_import_tiled_cbc(M, K, pad_elems, to.ctypes.data, ci.ctypes.data, bm.ctypes.data,
+                                     va.ctypes.data if va.size else None, va.size, ctypes.byref(h))
+    _check(st, "spdp_import_tiled_cbc")
+    return h.value
+
+
+def spdp_spmspv(h: int, x, rule: int, thr: float, y, mask=None, stream=None) -> None:
+    """x: fp16 CUDA [K]; y: fp16 or fp32 CUDA [M] (its dtype selects the output type)."""
+    import torch
+    ydt = SPDP_Y_F32 if y.dtype == torch.float32 else SPDP_Y_F16
+    if y.dtype not in (torch.float16, torch.float32) or x.dtype != torch.float16:
+        raise ValueError("x must be fp16 and y fp16 or fp32")
+    st = lib().spdp_spmspv(h, _dev_ptr(x, "x"), rule, float(thr), _dev_ptr(mask, "mask", True), _dev_ptr(y, "y"),
+                           ydt, _stream(stream))
+    _check(st, "spdp_spmspv")
+
+
+def spdp_spmspv_host(h: int, x_host, rule: int, thr: float, y_host, mask_host=None, stream=None) -> None:
+    """x_host / y_host: host arrays (NumPy or pinned torch CPU tensors); blocks until y_host is filled."""
+    ydt = SPDP_Y_F32 if str(y_host.dtype).endswith("float32") else SPDP_Y_F16
+    st = lib().spdp_spmspv_host(h, _host_ptr(x_host, "x_host"), rule, float(thr),
+                                _host_ptr(mask_host, "mask_host", True), _host_ptr(y_host, "y_host"), ydt,
+                                _stream(stream))
+    _check(st, "spdp_spmspv_host")
+
+
+def spdp_free(h) -> None:
+    _check(lib().spdp_free(h), "spdp_free")
+
+
+def spdp_get_info(h: int) -> spdp_info:
+    info = spdp_info()
+    _check(lib().spdp_get_info(h, ctypes.byref(info)), "spdp_get_info")
+    return info
+
+
+def spdp_export(h: int) -> dict:
+    """The four packed arrays as NumPy arrays (synchronous device-to-host copies)."""
+    info = spdp_get_info(h)
+    to = np.empty(info.NGT + 1, np.uint32)
+    ci = np.empty(info.NGT * 16, np.uint32)
+    bm = np.empty(info.NGT * 64, np.uint64)
+    va = np.empty(info.values_len, np.uint16)
+    st = lib().spdp_export(h, to.ctypes.data, ci.ctypes.data, bm.ctypes.data, va.ctypes.data if va.size else None)
+    _check(st, "spdp_export")
+    return dict(M=info.M, K=info.K, pad_elems=info.pad_elems, tileoffset=to, colinfo=ci, bitmap=bm, values=va,
+                nnz=info.nnz)
+
+
+def spdp_unpack(h: int, W_out, stream=None) -> None:
+    _check(lib().spdp_unpack(h, _dev_ptr(W_out, "W_out"), W_out.stride(0), _stream(stream)), "spdp_unpack")
+
+
+def spdp_active_columns(h: int, x, rule: int, thr: float, bitmask_out, count_out=None, mask=None, stream=None) -> None:
+    st = lib().spdp_active_columns(h, _dev_ptr(x, "x"), rule, float(thr), _dev_ptr(mask, "mask", True),
+                                   _dev_ptr(bitmask_out, "bitmask_out"), _dev_ptr(count_out, "count_out", True),
+                                   _stream(stream))
+    _check(st, "spdp_active_columns")
+
+
+def spdp_last_device_status(h: int) -> int:
+    v = ctypes.c_int(0)
+    _check(lib().spdp_last_device_status(h, ctypes.byref(v)), "spdp_last_device_status")
+    return v.value
+
+
+def spdp_set_num_ctas(h: int, num_ctas: int) -> None:
+    _check(lib().spdp_set_num_ctas(h, num_ctas), "spdp_set_num_ctas")
+
+
+def spdp_status_string(status: int) -> str:
+    return lib().spdp_status_string(status).decode()

@@ -1,0 +1,62 @@
+"""Parity at the benchmark's full sizes, in the launch configuration the benchmark times
+(default CTA count, fp16 y), against the C oracle: packed arrays and active set bit-exact, every
+output inside the tolerance."""
+import numpy as np
+import pytest
+
+from oracle import spdp_oracle as O
+from paper_2607_21985_b200 import workloads as WL
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+
+@pytest.fixture(scope="module")
+def S():
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    from paper_2607_21985_b200 import spdp
+    spdp.lib()
+    return spdp
+
+
+CASES = {
+    "c1": lambda: WL.config1(),
+    "c2": lambda: WL.config2(),
+    "c3": lambda: WL.config3(),
+    "c4": lambda: WL.config4(),
+    "c5_sp30_dp0": lambda: WL.config5(0, 0),
+    "c5_sp50_dp50": lambda: WL.config5(1, 2),
+    "c5_sp70_dp25": lambda: WL.config5(2, 1),
+    "c5_sp90_dp75": lambda: WL.config5(3, 3),
+}
+
+
+@pytest.mark.parametrize("name", list(CASES))
+def test_full_size_layer(S, c_oracle, name):
+    w = CASES[name]()
+    a = c_oracle.active(w.x, w.rule, w.thr)
+    want = c_oracle.pack(w.W)
+    y_ref, S_ref, _ = c_oracle.spmspv(w.W, w.x, a)
+    Wd = torch.from_numpy(w.W).cuda()
+    h = S.spdp_pack_tiled_cbc(Wd)
+    del Wd
+    try:
+        got = S.spdp_export(h)
+        for key in ("tileoffset", "colinfo", "bitmap", "values"):
+            assert np.array_equal(got[key], want[key]), key
+        xd = torch.from_numpy(w.x).cuda()
+        bits = torch.zeros((w.K + 31) // 32, dtype=torch.int32, device="cuda")
+        S.spdp_active_columns(h, xd, w.rule, w.thr, bits)
+        assert np.array_equal(bits.cpu().numpy().view(np.uint32), O.active_to_words(a))
+        for dt in (torch.float16, torch.float32):
+            y = torch.full((w.M,), float("nan"), dtype=dt, device="cuda")
+            S.spdp_spmspv(h, xd, w.rule, w.thr, y)
+            torch.cuda.synchronize()
+            assert S.spdp_last_device_status(h) == 0
+            err = np.abs(y.cpu().numpy().astype(np.float64) - y_ref)
+            tol = O.tolerance(S_ref)
+            assert np.all(err <= tol), f"{name}: worst error/tolerance {np.nanmax(err / tol):.3g}"
+    finally:
+        S.spdp_free(h)

@@ -1,0 +1,292 @@
+"""Parity of the CUDA library (through the C ABI) with the CPU oracle on the same seeded inputs.
+
+Bars: packed arrays and the active-column set bit-exact; every output within
+|y - y_ref| <= 1e-3 * sum_j |W_ij x_j| + 1e-5 (y widened to fp64, no re-rounding); exact
+equality where every partial sum is exactly representable.
+"""
+import numpy as np
+import pytest
+
+from oracle import spdp_oracle as O
+from paper_2607_21985_b200 import workloads as WL
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+
+
+@pytest.fixture(scope="module")
+def S():
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    from paper_2607_21985_b200 import spdp
+    spdp.lib()
+    return spdp
+
+
+def dev(a):
+    a = np.ascontiguousarray(a)
+    if a.dtype == np.uint32:
+        return torch.from_numpy(a.view(np.int32)).cuda()
+    return torch.from_numpy(a).cuda()
+
+
+def assert_same_packed(got, want):
+    for key in ("tileoffset", "colinfo", "bitmap", "values"):
+        assert got[key].dtype == want[key].dtype, key
+        assert got[key].shape == want[key].shape, key
+        assert np.array_equal(got[key], want[key]), key
+    assert got["nnz"] == want["nnz"]
+
+
+def gpu_spmspv(S, h, x, rule, thr, M, ydtype=torch.float32, mask_words=None):
+    xd = dev(x)
+    y = torch.full((M,), float("nan"), dtype=ydtype, device="cuda")        # poison: every entry must be written
+    md = dev(mask_words) if mask_words is not None else None
+    S.spdp_spmspv(h, xd, rule, thr, y, mask=md)
+    torch.cuda.synchronize()
+    assert S.spdp_last_device_status(h) == 0
+    return y.cpu().numpy().astype(np.float64)
+
+
+def gpu_active(S, h, x, rule, thr, K, mask_words=None):
+    bits = torch.full(((K + 31) // 32,), -1, dtype=torch.int32, device="cuda")
+    cnt = torch.full((1,), -7, dtype=torch.int32, device="cuda")
+    S.spdp_active_columns(h, dev(x), rule, thr, bits, cnt, mask=dev(mask_words) if mask_words is not None else None)
+    torch.cuda.synchronize()
+    return bits.cpu().numpy().view(np.uint32), int(cnt.item())
+
+
+def check_y(y, y_ref, S_ref):
+    err = np.abs(y - y_ref)
+    tol = O.tolerance(S_ref)
+    bad = np.flatnonzero(~(err <= tol))
+    assert bad.size == 0, f"{bad.size} outputs out of tolerance, worst ratio {np.nanmax(err / tol):.3g} at {bad[:5]}"
+    return float(np.max(err / tol))
+
+
+# ------------------------------------------------------------------------------------------
+# packer / unpacker: bit-exact
+# ------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("M,K,seed", [(256, 16, 1), (512, 48, 2), (1, 1, 3), (257, 17, 4), (300, 40, 5),
+                                      (1000, 200, 6), (2048, 272, 7)])
+def test_pack_bit_exact_and_unpack(S, M, K, seed):
+    W = WL.special_values_matrix(M, K, seed)
+    want = O.pack_fast(W)
+    h = S.spdp_pack_tiled_cbc(dev(W))
+    try:
+        got = S.spdp_export(h)
+        assert_same_packed(got, want)
+        info = S.spdp_get_info(h)
+        assert (info.M, info.K, info.nnz, info.values_len) == (M, K, want["nnz"], len(want["values"]))
+        assert info.packed_bytes == O.packed_bytes(want)
+        out = torch.full((M, K + 3), -1.0, dtype=torch.float16, device="cuda")[:, :K]   # ldw != K
+        S.spdp_unpack(h, out)
+        torch.cuda.synchronize()
+        assert np.array_equal(out.cpu().numpy().view(np.uint16), O.canon(W))
+    finally:
+        S.spdp_free(h)
+
+
+def test_pack_strided_input_and_storage_formula(S):
+    M, K = 512, 96
+    W = WL.special_values_matrix(M, K, 9)
+    big = torch.zeros((M, K + 24), dtype=torch.float16, device="cuda")
+    big[:, :K] = dev(W)
+    h8 = S.spdp_pack_tiled_cbc(big[:, :K])
+    h1 = S.spdp_pack_tiled_cbc(big[:, :K], pad_elems=1)
+    try:
+        assert_same_packed(S.spdp_export(h8), O.pack_fast(W))
+        got1 = S.spdp_export(h1)
+        assert_same_packed(got1, O.pack_fast(W, pad_elems=1))
+        nnz = int(np.count_nonzero(W.view(np.uint16) & 0x7FFF))
+        # Sec. 4.1 storage formula, exact when nothing is padded
+        assert S.spdp_get_info(h1).packed_bytes == O.storage_formula_bytes(M, K, nnz)
+        with pytest.raises(S.SpdpError, match="UNSUPPORTED_SHAPE"):
+            S.spdp_spmspv(h1, torch.zeros(K, dtype=torch.float16, device="cuda"), 0, 0.0,
+                          torch.zeros(M, dtype=torch.float32, device="cuda"))
+    finally:
+        S.spdp_free(h8)
+        S.spdp_free(h1)
+
+
+def test_pack_empty_and_full(S):
+    for fill in (0.0, 1.0):
+        W = np.full((512, 32), fill, np.float16)
+        h = S.spdp_pack_tiled_cbc(dev(W))
+        try:
+            assert_same_packed(S.spdp_export(h), O.pack_ref(W))
+        finally:
+            S.spdp_free(h)
+
+
+# ------------------------------------------------------------------------------------------
+# active-column set: bit-exact
+# ------------------------------------------------------------------------------------------
+def test_active_set_bit_exact(S):
+    K = 1000
+    rng = np.random.Generator(np.random.PCG64(11))
+    x = rng.standard_normal(K, dtype=np.float32).astype(np.float16)
+    thr = float(np.float16(0.5))
+    up, dn = np.nextafter(np.float16(0.5), np.float16(9)), np.nextafter(np.float16(0.5), np.float16(0))
+    x[:14] = np.asarray([0.0, -0.0, 0.5, -0.5, up, -up, dn, -dn, np.nan, np.inf, -np.inf, 6e-8, -6e-8, 65504], np.float16)
+    h = S.spdp_pack_tiled_cbc(dev(np.ones((256, K), np.float16)))
+    try:
+        for rule, t in ((O.DP_ABS_GT, thr), (O.DP_ABS_GT, 0.0), (O.DP_ABS_GT, -1.0), (O.DP_NONE, 0.0),
+                        (O.DP_ABS_GT, 1e30), (O.DP_ABS_GT, float("inf"))):
+            want = O.active_ref(x, rule, t)
+            bits, cnt = gpu_active(S, h, x, rule, t, K)
+            assert np.array_equal(bits, O.active_to_words(want)) and cnt == int(want.sum())
+        m = rng.random(K) < 0.3
+        bits, cnt = gpu_active(S, h, x, O.DP_MASK, 0.0, K, O.active_to_words(m))
+        assert np.array_equal(bits, O.active_to_words(m)) and cnt == int(m.sum())
+    finally:
+        S.spdp_free(h)
+
+
+# ------------------------------------------------------------------------------------------
+# spMspV against the oracle
+# ------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("M,K,sp,skip,seed", [
+    (256, 16, 0.5, 0.5, 1), (512, 64, 0.5, 0.0, 2), (300, 40, 0.3, 0.25, 3), (1, 1, 0.0, 0.0, 4),
+    (257, 17, 0.5, 0.5, 5), (1024, 1024, 0.5, 0.5, 6), (768, 4400, 0.7, 0.9, 7), (2304, 528, 0.9, 0.4, 8),
+    (4096, 272, 0.0, 0.1, 9), (256, 8192, 0.6, 0.5, 10)])
+@pytest.mark.parametrize("ydtype", ["f32", "f16"])
+def test_spmspv_matches_oracle(S, M, K, sp, skip, seed, ydtype):
+    rw, rx = WL._rngs(seed)
+    W = WL.prune_global_magnitude(WL.normal_weights(rw, M, K), sp).astype(np.float16)
+    x = rx.standard_normal(K, dtype=np.float32).astype(np.float16)
+    rule, thr = WL.skip_threshold(x, skip)
+    a = O.active_ref(x, rule, thr)
+    y_ref, S_ref = O.spmspv_ref(W, x, a)
+    h = S.spdp_pack_tiled_cbc(dev(W))
+    try:
+        bits, cnt = gpu_active(S, h, x, rule, thr, K)
+        assert np.array_equal(bits, O.active_to_words(a)) and cnt == int(a.sum())
+        yd = torch.float32 if ydtype == "f32" else torch.float16
+        y = gpu_spmspv(S, h, x, rule, thr, M, yd)
+        check_y(y, y_ref, S_ref)
+        y2 = gpu_spmspv(S, h, x, rule, thr, M, yd)
+        assert np.array_equal(y, y2)                                   # fixed summation order
+        for ctas in (1, 3, 37, 1000):                                  # other split-K layouts
+            S.spdp_set_num_ctas(h, ctas)
+            check_y(gpu_spmspv(S, h, x, rule, thr, M, yd), y_ref, S_ref)
+    finally:
+        S.spdp_free(h)
+
+
+def test_spmspv_exact_on_integers_and_powers_of_two(S):
+    """Every product and partial sum is exactly representable: the GPU must match exactly."""
+    rng = np.random.Generator(np.random.PCG64(21))
+    M, K = 700, 900
+    W = rng.integers(-8, 9, (M, K)).astype(np.float16)
+    W[rng.random((M, K)) < 0.6] = 0
+    x = rng.integers(-4, 5, K).astype(np.float16)
+    a = O.active_ref(x, O.DP_ABS_GT, 1.0)
+    y_ref, _ = O.spmspv_ref(W, x, a)
+    h = S.spdp_pack_tiled_cbc(dev(W))
+    try:
+        assert np.array_equal(gpu_spmspv(S, h, x, O.DP_ABS_GT, 1.0, M), y_ref)
+        Wp = (2.0 ** rng.integers(-6, 3, (M, K))).astype(np.float16) * rng.choice([-1, 1], (M, K)).astype(np.float16)
+        Wp[rng.random((M, K)) < 0.5] = 0
+        xp = (2.0 ** rng.integers(-3, 3, K)).astype(np.float16)
+        hp = S.spdp_pack_tiled_cbc(dev(Wp))
+        try:
+            yp_ref, _ = O.spmspv_ref(Wp, xp, np.ones(K, bool))
+            assert np.array_equal(gpu_spmspv(S, hp, xp, O.DP_NONE, 0.0, M), yp_ref)
+        finally:
+            S.spdp_free(hp)
+    finally:
+        S.spdp_free(h)
+
+
+def test_spmspv_degenerate_cases(S):
+    M, K = 600, 100
+    rng = np.random.Generator(np.random.PCG64(23))
+    W = (rng.standard_normal((M, K), dtype=np.float32) * 0.02).astype(np.float16)
+    W[:, 10:20] = 0                                  # empty columns
+    W[256:512, :] = 0                                # an empty row tile
+    x = rng.standard_normal(K, dtype=np.float32).astype(np.float16)
+    h = S.spdp_pack_tiled_cbc(dev(W))
+    try:
+        # nothing active: y is written as zeros
+        y = gpu_spmspv(S, h, x, O.DP_ABS_GT, 1e9, M)
+        assert not y.any()
+        y = gpu_spmspv(S, h, x, O.DP_MASK, 0.0, M, mask_words=np.zeros(4, np.uint32))
+        assert not y.any()
+        # a single active column; explicit mask rule
+        m = np.zeros(K, bool)
+        m[37] = True
+        y = gpu_spmspv(S, h, x, O.DP_MASK, 0.0, M, mask_words=O.active_to_words(m))
+        y_ref, S_ref = O.spmspv_ref(W, x, m)
+        check_y(y, y_ref, S_ref)
+        # NaN activation is active and propagates; Inf weight in a skipped column does not
+        W2 = W.copy()
+        W2[5, 50] = np.inf
+        x2 = x.copy()
+        x2[50] = 0.0
+        x2[60] = np.nan
+        h2 = S.spdp_pack_tiled_cbc(dev(W2))
+        try:
+            y = gpu_spmspv(S, h2, x2, O.DP_ABS_GT, 0.0, M)
+            nz60 = O.is_nonzero(W2[:, 60])
+            assert np.all(np.isnan(y[nz60])) and not np.isnan(y[~nz60]).any()
+        finally:
+            S.spdp_free(h2)
+    finally:
+        S.spdp_free(h)
+
+
+def test_imported_oracle_arrays_give_same_result(S):
+    w = WL.config1(768, 640, seed=4)
+    p = O.pack_fast(w.W)
+    h_imp = S.spdp_import_tiled_cbc(w.M, w.K, p["tileoffset"], p["colinfo"], p["bitmap"], p["values"])
+    h_gpu = S.spdp_pack_tiled_cbc(dev(w.W))
+    try:
+        assert_same_packed(S.spdp_export(h_imp), p)
+        y1 = gpu_spmspv(S, h_imp, w.x, w.rule, w.thr, w.M)
+        y2 = gpu_spmspv(S, h_gpu, w.x, w.rule, w.thr, w.M)
+        assert np.array_equal(y1, y2)
+        bad = p["colinfo"].copy()
+        bad[3] += 1
+        with pytest.raises(S.SpdpError, match="INVALID_ARG"):
+            S.spdp_import_tiled_cbc(w.M, w.K, p["tileoffset"], bad, p["bitmap"], p["values"])
+    finally:
+        S.spdp_free(h_imp)
+        S.spdp_free(h_gpu)
+
+
+def test_host_vector_entry_point(S):
+    w = WL.config2(1024, 512, seed=6)
+    a = O.active_ref(w.x, w.rule, w.thr)
+    y_ref, S_ref = O.spmspv_ref(w.W, w.x, a)
+    h = S.spdp_pack_tiled_cbc(dev(w.W))
+    try:
+        xh = torch.from_numpy(w.x.copy()).pin_memory()
+        for dt in (torch.float16, torch.float32):
+            yh = torch.full((w.M,), float("nan"), dtype=dt).pin_memory()
+            S.spdp_spmspv_host(h, xh, w.rule, w.thr, yh)
+            check_y(yh.numpy().astype(np.float64), y_ref, S_ref)
+        yn = np.full(w.M, np.nan, np.float32)
+        S.spdp_spmspv_host(h, w.x, O.DP_MASK, 0.0, yn, mask_host=O.active_to_words(a))
+        check_y(yn.astype(np.float64), y_ref, S_ref)
+    finally:
+        S.spdp_free(h)
+
+
+@pytest.mark.parametrize("make", [lambda: WL.config1(1024, 1024), lambda: WL.config2(1536, 1024),
+                                  lambda: WL.config3(1024, 2752), lambda: WL.config4(3584, 1024),
+                                  lambda: WL.config5(0, 0, 1024, 1024), lambda: WL.config5(3, 3, 1024, 1024)])
+def test_scaled_down_benchmark_layers(S, make):
+    w = make()
+    a = O.active_ref(w.x, w.rule, w.thr)
+    y_ref, S_ref = O.spmspv_ref(w.W, w.x, a)
+    h = S.spdp_pack_tiled_cbc(dev(w.W))
+    try:
+        assert_same_packed(S.spdp_export(h), O.pack_fast(w.W))
+        bits, _ = gpu_active(S, h, w.x, w.rule, w.thr, w.K)
+        assert np.array_equal(bits, O.active_to_words(a))
+        check_y(gpu_spmspv(S, h, w.x, w.rule, w.thr, w.M, torch.float16), y_ref, S_ref)
+        check_y(gpu_spmspv(S, h, w.x, w.rule, w.thr, w.M, torch.float32), y_ref, S_ref)
+    finally:
+        S.spdp_free(h)

@@ -70,10 +70,8 @@ spdp_status build_partition(spdp_matrix* h, int num_ctas) {
     std::vector<uint32_t> begin(P + 1);
     for (int p = 0; p <= P; ++p) begin[p] = static_cast<uint32_t>((static_cast<__int128>(NGT) * p) / P);
     std::vector<int32_t> first(R, -1), nseg(R, 0);
-    int max_segs = 1;
     for (int p = 0; p < P; ++p) {
         const int64_t r0 = begin[p] / C, r1 = (static_cast<int64_t>(begin[p + 1]) - 1) / C;
-        max_segs = max_segs > static_cast<int>(r1 - r0 + 1) ? max_segs : static_cast<int>(r1 - r0 + 1);
         for (int64_t r = r0; r <= r1; ++r) {
             if (first[r] < 0) first[r] = p;
             ++nseg[r];
@@ -85,8 +83,7 @@ spdp_status build_partition(spdp_matrix* h, int num_ctas) {
     cudaFree(h->workspace);     h->workspace = nullptr;
     cudaFree(h->row_counter);   h->row_counter = nullptr;
     h->num_ctas = P;
-    h->max_segs = max_segs;
-    h->workspace_bytes = static_cast<int64_t>(P) * max_segs * kTileM * sizeof(float);
+    h->workspace_bytes = static_cast<int64_t>(P) * 2 * kTileM * sizeof(float);   // two slots per CTA
     SPDP_CUDA_TRY(cudaMalloc(&h->cta_begin, (P + 1) * sizeof(uint32_t)));
     SPDP_CUDA_TRY(cudaMalloc(&h->row_first_cta, R * sizeof(int32_t)));
     SPDP_CUDA_TRY(cudaMalloc(&h->row_nseg, R * sizeof(int32_t)));

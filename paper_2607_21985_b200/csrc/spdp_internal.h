@@ -34,11 +34,10 @@ struct spdp_matrix {
 
     // Work partition of one spmspv launch: CTA p owns GTiles [cta_begin[p], cta_begin[p+1]).
     int num_ctas;           // P
-    int max_segs;           // most row tiles one CTA's range touches
     uint32_t* cta_begin;    // device [P+1]
     int32_t* row_first_cta; // device [R]: first CTA whose range touches row tile r
     int32_t* row_nseg;      // device [R]: number of CTAs whose range touches row tile r
-    float* workspace;       // device [P*max_segs*256] split-K partial sums
+    float* workspace;       // device [P*2*256] split-K partial sums (two slots per CTA)
     unsigned* row_counter;  // device [R] arrivals per row tile (self-resetting)
     int* status_word;       // device [1]
     int64_t workspace_bytes;

@@ -7,7 +7,9 @@
 // fp32 partial sums.  A row tile fed by one segment is written to y directly; otherwise the
 // partials go to the handle's workspace (the paper's ReductionWorkspace) and the CTA that
 // arrives last at the row tile's counter adds them in segment order -- no CTA ever waits for
-// another, and the order of the additions is fixed.
+// another, and the order of the additions is fixed.  Only the first and the last segment of a
+// CTA can share their row tile with another CTA, so a CTA owns two workspace slots: slot 0 for
+// the row tile its range starts in, slot 1 for any later one.
 #include "spdp_internal.h"
 
 namespace spdp {
@@ -33,7 +35,6 @@ struct Params {
     const int32_t* row_first_cta;
     const int32_t* row_nseg;
     float* workspace;
-    int max_segs;
     unsigned* row_counter;
     int* status;
 };
@@ -158,7 +159,7 @@ spmspv_kernel(const Params p) {
         if (nseg == 1) {
             if (t < kTileM && row < p.M) store_y(p.y, p.ydt, row, part);
         } else {
-            float* mine = p.workspace + (static_cast<int64_t>(blockIdx.x) * p.max_segs + (r - r_first)) * kTileM;
+            float* mine = p.workspace + (static_cast<int64_t>(blockIdx.x) * 2 + (r != r_first)) * kTileM;
             if (t < kTileM) __stcg(mine + t, part);
             __threadfence();
             __syncthreads();
@@ -174,8 +175,8 @@ spmspv_kernel(const Params p) {
                     float sum = 0.f;
                     for (int s = 0; s < nseg; ++s) {
                         const int q = q0 + s;
-                        const int ls = r - static_cast<int>(p.cta_begin[q] / p.C);
-                        sum += __ldcg(p.workspace + (static_cast<int64_t>(q) * p.max_segs + ls) * kTileM + t);
+                        const int slot = (r != static_cast<int>(p.cta_begin[q] / p.C));
+                        sum += __ldcg(p.workspace + (static_cast<int64_t>(q) * 2 + slot) * kTileM + t);
                     }
                     store_y(p.y, p.ydt, row, sum);
                 }
@@ -222,7 +223,6 @@ spdp_status launch_spmspv(const spdp_matrix* h, const __half* x, int rule, float
     p.row_first_cta = h->row_first_cta;
     p.row_nseg = h->row_nseg;
     p.workspace = h->workspace;
-    p.max_segs = h->max_segs;
     p.row_counter = h->row_counter;
     p.status = h->status_word;
     spmspv_kernel<<<h->num_ctas, kThreads, 0, s>>>(p);

@@ -196,7 +196,10 @@ def spdp_export(h: int) -> dict:
 
 
 def spdp_unpack(h: int, W_out, stream=None) -> None:
-    _check(lib().spdp_unpack(h, _dev_ptr(W_out, "W_out"), W_out.stride(0), _stream(stream)), "spdp_unpack")
+    """W_out: fp16 CUDA tensor [M, K] with unit column stride (row stride = ldw)."""
+    if not W_out.is_cuda or W_out.dim() != 2 or W_out.stride(1) != 1:
+        raise ValueError("W_out must be a 2-D fp16 CUDA tensor with unit column stride")
+    _check(lib().spdp_unpack(h, W_out.data_ptr(), W_out.stride(0), _stream(stream)), "spdp_unpack")
 
 
 def spdp_active_columns(h: int, x, rule: int, thr: float, bitmask_out, count_out=None, mask=None, stream=None) -> None:

@@ -126,6 +126,32 @@ SPDP_API spdp_status spdp_spmspv(spdp_handle h, const void* x_dev, spdp_dp_rule 
 SPDP_API spdp_status spdp_spmspv_host(spdp_handle h, const void* x_host, spdp_dp_rule rule, float thr,
                              const void* mask_host, void* y_host, spdp_ydtype ydt, void* stream);
 
+/* The same product for callers that must not allocate (the paper has no counterpart: this entry
+ * point exists for the library's users, not for the method).  Some hosts of this code cannot
+ * call cudaMalloc at all: a serving process that hands all device memory to its own arena at
+ * start-up, an embedding that forbids driver allocations after initialisation, a caller that
+ * already holds the four Tiled-CBC arrays in memory it manages.  For them nothing here creates a
+ * handle; the caller passes the packed arrays (device pointers, laid out as spdp_info describes,
+ * 16-byte column padding), x, the DP rule and y, exactly as for spdp_spmspv.
+ *
+ * What spdp_spmspv keeps in handle-owned allocations (CTA ranges, per-row-tile tables, arrival
+ * counters, split-K partial sums) lives in ONE fixed device array inside the library, about
+ * 0.6 MB, present on every GPU that loads the library until the process exits.  Limits: at most
+ * 4096 row tiles (M <= 1,048,576); larger shapes return SPDP_ERR_UNSUPPORTED_SHAPE.  At most 256
+ * CTAs are launched.  The call enqueues a small set-up kernel (which also clears the counters the
+ * previous call left behind) and the spMspV kernel on `stream`; it calls no cudaMalloc, cudaFree or
+ * allocating library routine.
+ *
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
+ * that device current) and the SM count; make that first call outside any stream capture.
+ * Every call on a device shares the one array: two calls that can overlap on the GPU (different
+ * streams without ordering, or two host threads) race on it and give wrong sums; order them.
+ * Results equal spdp_spmspv's for the same CTA count. */
+SPDP_API spdp_status spdp_spmspv_noalloc(const void* tileoffset_dev, const void* colinfo_dev,
+                                const void* bitmap_dev, const void* values_dev, int64_t M, int64_t K,
+                                const void* x_dev, spdp_dp_rule rule, float thr, const void* mask_dev,
+                                void* y_dev, spdp_ydtype ydt, void* stream);
+
 /* Release the handle and everything it owns.  spdp_free(NULL) is SPDP_OK. */
 SPDP_API spdp_status spdp_free(spdp_handle h);
 

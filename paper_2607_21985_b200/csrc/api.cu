@@ -204,6 +204,27 @@ spdp_status spdp_spmspv(spdp_handle h, const void* x_dev, spdp_dp_rule rule, flo
                          static_cast<const uint32_t*>(mask_dev), y_dev, ydt, static_cast<cudaStream_t>(stream));
 }
 
+spdp_status spdp_spmspv_noalloc(const void* tileoffset_dev, const void* colinfo_dev, const void* bitmap_dev,
+                                const void* values_dev, int64_t M, int64_t K, const void* x_dev,
+                                spdp_dp_rule rule, float thr, const void* mask_dev, void* y_dev,
+                                spdp_ydtype ydt, void* stream) {
+    if (tileoffset_dev == nullptr || colinfo_dev == nullptr || bitmap_dev == nullptr || values_dev == nullptr ||
+        x_dev == nullptr || y_dev == nullptr)
+        return SPDP_ERR_INVALID_ARG;
+    if (M < 1 || K < 1) return SPDP_ERR_UNSUPPORTED_SHAPE;
+    if (!rule_ok(rule) || (ydt != SPDP_Y_F16 && ydt != SPDP_Y_F32)) return SPDP_ERR_INVALID_ARG;
+    if (rule == SPDP_DP_MASK && mask_dev == nullptr) return SPDP_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(values_dev) & 15u) || (reinterpret_cast<uintptr_t>(bitmap_dev) & 7u) ||
+        (reinterpret_cast<uintptr_t>(tileoffset_dev) & 3u) || (reinterpret_cast<uintptr_t>(colinfo_dev) & 3u) ||
+        (reinterpret_cast<uintptr_t>(x_dev) & 1u) || (reinterpret_cast<uintptr_t>(mask_dev) & 3u) ||
+        (reinterpret_cast<uintptr_t>(y_dev) & (ydt == SPDP_Y_F32 ? 3u : 1u)))
+        return SPDP_ERR_INVALID_ARG;
+    return launch_spmspv_noalloc(static_cast<const uint32_t*>(tileoffset_dev), static_cast<const uint32_t*>(colinfo_dev),
+                                 static_cast<const uint64_t*>(bitmap_dev), static_cast<const __half*>(values_dev), M, K,
+                                 static_cast<const __half*>(x_dev), rule, thr, static_cast<const uint32_t*>(mask_dev),
+                                 y_dev, ydt, static_cast<cudaStream_t>(stream));
+}
+
 spdp_status spdp_spmspv_host(spdp_handle h, const void* x_host, spdp_dp_rule rule, float thr,
                              const void* mask_host, void* y_host, spdp_ydtype ydt, void* stream) {
     if (!valid(h) || x_host == nullptr || y_host == nullptr) return SPDP_ERR_INVALID_ARG;

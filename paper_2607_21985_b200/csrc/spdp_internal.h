@@ -71,6 +71,9 @@ spdp_status unpack_device(const spdp_matrix* h, __half* W, int64_t ldw, cudaStre
 // spmspv.cu
 spdp_status launch_spmspv(const spdp_matrix* h, const __half* x, int rule, float thr,
                           const uint32_t* mask, void* y, int ydt, cudaStream_t s);
+spdp_status launch_spmspv_noalloc(const uint32_t* tileoffset, const uint32_t* colinfo, const uint64_t* bitmap,
+                                  const __half* values, int64_t M, int64_t K, const __half* x, int rule,
+                                  float thr, const uint32_t* mask, void* y, int ydt, cudaStream_t s);
 spdp_status launch_active_columns(const spdp_matrix* h, const __half* x, int rule, float thr,
                                   const uint32_t* mask, uint32_t* bits, int* count, cudaStream_t s);
 

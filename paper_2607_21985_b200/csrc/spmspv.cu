@@ -10,6 +10,8 @@
 // another, and the order of the additions is fixed.  Only the first and the last segment of a
 // CTA can share their row tile with another CTA, so a CTA owns two workspace slots: slot 0 for
 // the row tile its range starts in, slot 1 for any later one.
+#include <mutex>
+
 #include "spdp_internal.h"
 
 namespace spdp {
@@ -200,6 +202,42 @@ __global__ void active_columns_kernel(const __half* __restrict__ x, int K, int r
     }
 }
 
+
+// ---- allocation-free variant: scratch in a file-scope device array --------------------------
+// Everything spdp_spmspv keeps in handle-owned allocations (the CTA ranges, the per-row-tile
+// tables, the arrival counters, the split-K partial sums) lives here instead, so the entry point
+// below never allocates.  One copy per device that loads the library, held until exit.
+constexpr int kNoAllocMaxCtas = 256;
+constexpr int kNoAllocMaxRowTiles = 4096;          // M <= 1,048,576
+
+struct NoAllocScratch {
+    uint32_t cta_begin[kNoAllocMaxCtas + 1];
+    int32_t row_first_cta[kNoAllocMaxRowTiles];
+    int32_t row_nseg[kNoAllocMaxRowTiles];
+    unsigned row_counter[kNoAllocMaxRowTiles];
+    int status;
+    float workspace[kNoAllocMaxCtas * 2 * kTileM];
+};
+
+static __device__ __align__(256) unsigned char g_noalloc_scratch[sizeof(NoAllocScratch)];
+
+// Fills the partition tables for P CTAs and zeroes what a call expects to start at zero (the
+// array keeps whatever the previous call left).
+__global__ void noalloc_setup_kernel(NoAllocScratch* sc, int64_t NGT, int64_t C, int R, int P) {
+    for (int p = threadIdx.x; p <= P; p += blockDim.x)
+        sc->cta_begin[p] = static_cast<uint32_t>((static_cast<unsigned long long>(NGT) * p) / P);
+    for (int r = threadIdx.x; r < R; r += blockDim.x) {
+        // the CTA whose range holds GTile s is ceil((s+1)*P/NGT) - 1
+        const unsigned long long s0 = static_cast<unsigned long long>(r) * C, s1 = s0 + C - 1;
+        const int first = static_cast<int>(((s0 + 1) * P + NGT - 1) / NGT) - 1;
+        const int last = static_cast<int>(((s1 + 1) * P + NGT - 1) / NGT) - 1;
+        sc->row_first_cta[r] = first;
+        sc->row_nseg[r] = last - first + 1;
+        sc->row_counter[r] = 0;
+    }
+    if (threadIdx.x == 0) sc->status = 0;
+}
+
 }  // namespace
 
 spdp_status launch_spmspv(const spdp_matrix* h, const __half* x, int rule, float thr,
@@ -226,6 +264,63 @@ spdp_status launch_spmspv(const spdp_matrix* h, const __half* x, int rule, float
     p.row_counter = h->row_counter;
     p.status = h->status_word;
     spmspv_kernel<<<h->num_ctas, kThreads, 0, s>>>(p);
+    SPDP_CUDA_TRY(cudaGetLastError());
+    return SPDP_OK;
+}
+
+spdp_status launch_spmspv_noalloc(const uint32_t* tileoffset, const uint32_t* colinfo, const uint64_t* bitmap,
+                                  const __half* values, int64_t M, int64_t K, const __half* x, int rule,
+                                  float thr, const uint32_t* mask, void* y, int ydt, cudaStream_t s) {
+    constexpr int kMaxDevices = 64;
+    static NoAllocScratch* scratch_of[kMaxDevices] = {};
+    static int sm_count_of[kMaxDevices] = {};
+    static std::mutex mu;
+    const int64_t R = (M + kTileM - 1) / kTileM, C = (K + kTileK - 1) / kTileK, NGT = R * C;
+    if (R > kNoAllocMaxRowTiles || NGT >= (int64_t(1) << 31) / kTileK) return SPDP_ERR_UNSUPPORTED_SHAPE;
+    int dev = 0;
+    SPDP_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return SPDP_ERR_UNSUPPORTED_SHAPE;
+    NoAllocScratch* sc = nullptr;
+    int sms = 0;
+    {
+        // Once per device, with that device current: the array's name is only a host-side stand-in,
+        // so ask the runtime for the device address and hand THAT to the kernels.
+        std::lock_guard<std::mutex> lock(mu);
+        if (scratch_of[dev] == nullptr) {
+            void* ptr = nullptr;
+            SPDP_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_noalloc_scratch));
+            SPDP_CUDA_TRY(cudaDeviceGetAttribute(&sm_count_of[dev], cudaDevAttrMultiProcessorCount, dev));
+            scratch_of[dev] = static_cast<NoAllocScratch*>(ptr);
+        }
+        sc = scratch_of[dev];
+        sms = sm_count_of[dev];
+    }
+    int P = sms < kNoAllocMaxCtas ? sms : kNoAllocMaxCtas;
+    if (P > NGT) P = static_cast<int>(NGT);
+    noalloc_setup_kernel<<<1, 256, 0, s>>>(sc, NGT, C, static_cast<int>(R), P);
+    SPDP_CUDA_TRY(cudaGetLastError());
+    Params p;
+    p.tileoffset = tileoffset;
+    p.colinfo = colinfo;
+    p.bitmap = bitmap;
+    p.values = values;
+    p.x = x;
+    p.mask = mask;
+    p.y = y;
+    p.thr = thr;
+    p.rule = rule;
+    p.ydt = ydt;
+    p.M = static_cast<int>(M);
+    p.K = static_cast<int>(K);
+    p.R = static_cast<int>(R);
+    p.C = static_cast<int>(C);
+    p.cta_begin = sc->cta_begin;            // addresses inside the device array (no host dereference)
+    p.row_first_cta = sc->row_first_cta;
+    p.row_nseg = sc->row_nseg;
+    p.workspace = sc->workspace;
+    p.row_counter = sc->row_counter;
+    p.status = &sc->status;
+    spmspv_kernel<<<P, kThreads, 0, s>>>(p);
     SPDP_CUDA_TRY(cudaGetLastError());
     return SPDP_OK;
 }

@@ -27,7 +27,7 @@ SPDP_Y_F16, SPDP_Y_F32 = 0, 1
 
 EXPORTS = (
     "spdp_pack_tiled_cbc", "spdp_pack_tiled_cbc_ex", "spdp_import_tiled_cbc", "spdp_spmspv",
-    "spdp_spmspv_host", "spdp_free", "spdp_get_info", "spdp_export", "spdp_unpack",
+    "spdp_spmspv_host", "spdp_spmspv_noalloc", "spdp_free", "spdp_get_info", "spdp_export", "spdp_unpack",
     "spdp_active_columns", "spdp_last_device_status", "spdp_set_num_ctas", "spdp_last_cuda_error",
     "spdp_status_string",
 )
@@ -65,6 +65,7 @@ def lib():
         L.spdp_import_tiled_cbc.argtypes = [i64, i64, ci, vp, vp, vp, vp, i64, ctypes.POINTER(vp)]
         L.spdp_spmspv.argtypes = [vp, vp, ci, cf, vp, vp, ci, vp]
         L.spdp_spmspv_host.argtypes = [vp, vp, ci, cf, vp, vp, ci, vp]
+        L.spdp_spmspv_noalloc.argtypes = [vp, vp, vp, vp, i64, i64, vp, ci, cf, vp, vp, ci, vp]
         L.spdp_free.argtypes = [vp]
         L.spdp_get_info.argtypes = [vp, ctypes.POINTER(spdp_info)]
         L.spdp_export.argtypes = [vp, vp, vp, vp, vp]
@@ -170,6 +171,22 @@ def spdp_spmspv_host(h: int, x_host, rule: int, thr: float, y_host, mask_host=No
                                 _host_ptr(mask_host, "mask_host", True), _host_ptr(y_host, "y_host"), ydt,
                                 _stream(stream))
     _check(st, "spdp_spmspv_host")
+
+
+def spdp_spmspv_noalloc(tileoffset, colinfo, bitmap, values, M: int, K: int, x, rule: int, thr: float, y,
+                        mask=None, stream=None) -> None:
+    """The allocation-free call: the four packed arrays are CUDA tensors (or raw device addresses)
+    owned by the caller; scratch lives in a fixed array inside the library.  For callers that
+    cannot let the library allocate device memory; see spdp.h for the limits and the sharing rule."""
+    import torch
+    ydt = SPDP_Y_F32 if y.dtype == torch.float32 else SPDP_Y_F16
+    if y.dtype not in (torch.float16, torch.float32) or x.dtype != torch.float16:
+        raise ValueError("x must be fp16 and y fp16 or fp32")
+    ptr = lambda t, n: t if isinstance(t, int) else _dev_ptr(t, n)
+    st = lib().spdp_spmspv_noalloc(ptr(tileoffset, "tileoffset"), ptr(colinfo, "colinfo"), ptr(bitmap, "bitmap"),
+                                   ptr(values, "values"), M, K, _dev_ptr(x, "x"), rule, float(thr),
+                                   _dev_ptr(mask, "mask", True), _dev_ptr(y, "y"), ydt, _stream(stream))
+    _check(st, "spdp_spmspv_noalloc")
 
 
 def spdp_free(h) -> None:

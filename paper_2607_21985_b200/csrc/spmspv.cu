@@ -17,16 +17,14 @@
 namespace spdp {
 namespace {
 
-constexpr int kConsumers = 12;             // consumer (decode) warps per CTA; one more warp feeds them
-constexpr int kDepth = 4;                  // ring stages owned by each consumer warp
-constexpr int kStages = kConsumers * kDepth;
-constexpr int kGroup = 4;                  // active column tiles per ring stage (one consumer work unit)
+constexpr int kWarps = 16;                 // warps per CTA; every warp fetches and decodes its own column tiles
+constexpr int kDepth = 3;                  // groups a warp keeps in flight
+constexpr int kGroup = 4;                  // active column tiles per group (one fetch / decode unit of a warp)
 constexpr int kSlotBytes = 2 * kTileM;     // a column tile's values: at most 256 fp16
 constexpr int kStageBytes = kGroup * kSlotBytes;
-constexpr int kThreads = (kConsumers + 1) * 32;
+constexpr int kThreads = kWarps * 32;
 constexpr int kChunkCols = 8192;           // columns handled between two pipeline drains
 constexpr int kChunkGT = kChunkCols / kTileK;
-constexpr unsigned kSpinLimit = 1u << 20;  // bound of every mbarrier wait
 
 struct Params {
     const uint32_t* tileoffset;
@@ -49,18 +47,15 @@ struct Params {
 };
 
 struct __align__(128) Smem {
-    unsigned char ring[kStages * kStageBytes];          // values of the column tiles in flight
+    unsigned char ring[kWarps][kDepth][kStageBytes];    // values of the column tiles in flight, per warp
+    uint32_t bmring[kWarps][kDepth][32];                // their bitmap words (8 words x 4 column tiles)
     uint32_t colinfo[kChunkCols];                       // ColInfo words of the chunk's GTiles
     uint32_t tileoff[kChunkGT + 1];                     // TileOffset of the chunk's GTiles
     uint32_t ent[kChunkCols];                           // active list: (column in chunk) << 16 | x bits
-    uint32_t bmring[kConsumers][kDepth][32];            // bitmap words of a warp's next groups
-    float red[kConsumers][kTileM];
+    float red[kWarps][kTileM];
     uint32_t group_mask[kChunkCols / 32];
     uint32_t group_base[kChunkCols / 32 + 1];
-    unsigned long long full[kStages];                   // values of a stage have landed
-    unsigned long long empty[kStages];                  // the stage's consumer is done with it
     int is_last;
-    int abort;                                          // a bounded wait expired: stop waiting anywhere
 };
 
 // DP test of Sec. 4.2 step (3): magnitude against the threshold; NOT(|x| <= thr) keeps NaN.
@@ -78,37 +73,10 @@ __device__ __forceinline__ void store_y(void* y, int ydt, int64_t i, float v) {
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, unsigned count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("{\n .reg .b64 st;\n mbarrier.arrive.shared::cta.b64 st, [%0];\n}" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, unsigned bytes) {
-    asm volatile("{\n .reg .b64 st;\n mbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1;\n}" ::"r"(bar), "r"(bytes)
-                 : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, unsigned parity) {
-    unsigned ok;
-    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
-                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait: gives up after kSpinLimit polls (or as soon as another thread gave up), records
-// SPDP_ERR_TIMEOUT in the device status word and lets the kernel run to its end.
-__device__ __forceinline__ void mbar_wait(uint32_t bar, unsigned parity, volatile int* abort_flag, int* status) {
-    for (unsigned it = 0; it < kSpinLimit; ++it) {
-        if (mbar_try_wait(bar, parity)) return;
-        if (*abort_flag) return;
-    }
-    *abort_flag = 1;
-    atomicExch(status, static_cast<int>(SPDP_ERR_TIMEOUT));
-}
-// 1-D bulk copy global -> shared, completion counted in bytes on an mbarrier (no multicast).
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, unsigned bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+// Asynchronous global -> shared copies (Sec. 4.2.3: 128-bit per thread); `on` = false copies nothing.
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool on) {
+    asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %2, 0;\n @p cp.async.cg.shared.global [%0], [%1], 16;\n}"
+                 ::"r"(dst), "l"(src), "r"(static_cast<int>(on)) : "memory");
 }
 __device__ __forceinline__ void cp_async4(uint32_t dst, const void* src) {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
@@ -117,24 +85,21 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-__device__ __forceinline__ unsigned short lds_u16(uint32_t addr) {
-    unsigned short v;
-    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(addr));
-    return v;
-}
 // acc += w * x with fp16 operands and an fp32 accumulator: the product of two fp16 is exact in fp32.
 __device__ __forceinline__ void fma_f16(float& acc, unsigned short w, unsigned short x) {
     asm("fma.rn.f32.f16 %0, %1, %2, %0;" : "+f"(acc) : "h"(w), "h"(x));
 }
 
-// One CTA = kConsumers decode warps + 1 producer warp.  Per chunk of its GTile range:
-//   (1) all warps: ColInfo / TileOffset of the chunk to shared memory, active-column list from x
-//       (ballots + prefix sums), Sec. 4.2 steps (1)-(3);
-//   (2) producer warp: one bulk copy per active column tile (its padded values, straight from
-//       Values) into a ring of kStages stages of kGroup column tiles, mbarrier-tracked;
-//       consumer warps: prefetch the column tiles' bitmap words with 4-byte async copies, wait
-//       for their stage, decode (lane = 4 consecutive rows; rank = set bits before, Sec. 4.2.1)
-//       and accumulate in fp32 registers;
+// One persistent CTA per GTile range; every warp runs its own fetch -> decode pipeline.
+// Per chunk of the range:
+//   (1) all warps: ColInfo / TileOffset of the chunk to shared memory and the active-column list
+//       from x (ballots + prefix sums) -- Sec. 4.2 steps (1)-(3);
+//   (2) each warp takes groups of kGroup active column tiles round-robin.  It keeps kDepth
+//       groups in flight: the padded values of a column tile arrive with 16-byte asynchronous
+//       copies (lane = one 16-byte piece of one of the group's tiles), its 8 bitmap words with
+//       4-byte ones; inactive columns are never touched.  Decode (Sec. 4.2.1): lane owns 4
+//       consecutive rows of a half column tile, rank = set bits before them, values read from
+//       shared memory, fp32 accumulation in registers;
 //   (3) segment end: cross-warp row reduction, split-K combine, store.
 __global__ void __launch_bounds__(kThreads, 1)
 spmspv_kernel(const Params p) {
@@ -142,26 +107,14 @@ spmspv_kernel(const Params p) {
     Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
 
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
-    const bool is_producer = (warp == kConsumers);
     const int64_t g_begin = p.cta_begin[blockIdx.x], g_end = p.cta_begin[blockIdx.x + 1];
     const int r_first = static_cast<int>(g_begin / p.C);
-    volatile int* abort_flag = &sm.abort;
 
-    if (t == 0) {
-        for (int s = 0; s < kStages; ++s) {
-            mbar_init(smem_u32(&sm.full[s]), 1);
-            mbar_init(smem_u32(&sm.empty[s]), 1);
-        }
-        sm.abort = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    __syncthreads();
-
-    const uint32_t ring_base = smem_u32(sm.ring);
-    unsigned gbase = 0;                 // groups handed out so far (ring positions keep running)
     const unsigned sh = 4u * (lane & 7);            // my nibble inside a 32-bit bitmap word
     const unsigned lt_mask = (1u << sh) - 1u;
-    const int lgrp = lane >> 3;                     // which of the 4 words of a half column tile
+    const int lgrp = lane >> 3;                     // which item of a group I fetch for / which word I decode
+    const unsigned char* bm8 = reinterpret_cast<const unsigned char*>(p.bitmap);
+    const unsigned char* val8 = reinterpret_cast<const unsigned char*>(p.values);
 
     for (int64_t g0 = g_begin; g0 < g_end;) {
         const int r = static_cast<int>(g0 / p.C);
@@ -170,7 +123,7 @@ spmspv_kernel(const Params p) {
         const int c_hi = static_cast<int>(c_end < p.C ? c_end : p.C);
         g0 += c_hi - c_lo;
 
-        float acc[8];                   // rows 4*lane+k (k<4) and 128+4*lane+k-4 of the row tile
+        float acc[8];                   // rows 4*lane+k (k<4) and 128+4*lane+(k-4) of the row tile
 #pragma unroll
         for (int k = 0; k < 8; ++k) acc[k] = 0.f;
 
@@ -185,7 +138,7 @@ spmspv_kernel(const Params p) {
             // ---- (1) metadata of the chunk and its active-column list ----
             for (int i = t; i < ngt * kTileK; i += kThreads) sm.colinfo[i] = __ldg(p.colinfo + gt0 * kTileK + i);
             for (int i = t; i < ngt; i += kThreads) sm.tileoff[i] = __ldg(p.tileoffset + gt0 + i);
-            for (int q = warp; q < ngroups32; q += kConsumers + 1) {
+            for (int q = warp; q < ngroups32; q += kWarps) {
                 const int j = j0 + q * 32 + lane;
                 bool a = false;
                 if (j < j_hi) a = column_active(p.rule, p.thr, p.mask, j, p.x[j]);
@@ -210,7 +163,7 @@ spmspv_kernel(const Params p) {
                 if (lane == 0) sm.group_base[ngroups32] = run;
             }
             __syncthreads();
-            for (int q = warp; q < ngroups32; q += kConsumers + 1) {
+            for (int q = warp; q < ngroups32; q += kWarps) {
                 const unsigned m = sm.group_mask[q];
                 if ((m >> lane) & 1u) {
                     const int jj = q * 32 + lane;
@@ -222,112 +175,87 @@ spmspv_kernel(const Params p) {
             const int nact = static_cast<int>(sm.group_base[ngroups32]);
             const int ngroups = (nact + kGroup - 1) / kGroup;
 
-            if (is_producer) {
-                // ---- (2a) producer: lane = one column tile, 8 ring stages per pass ----
-                for (int b = 0; b * 8 < ngroups; ++b) {
-                    const int lq = b * 8 + (lane >> 2);
-                    const int item = lq * kGroup + (lane & 3);
-                    const unsigned G = gbase + lq;
-                    const unsigned s = G % kStages, use = G / kStages;
-                    unsigned bytes = 0;
-                    const __half* src = nullptr;
+            // ---- (2) per-warp fetch / decode pipeline over groups warp, warp + kWarps, ... ----
+            // fetch(i): start the copies of my i-th group into ring position i % kDepth
+            auto fetch = [&](int i) {
+                const int lq = warp + i * kWarps;
+                if (lq < ngroups) {
+                    const int d = i % kDepth;
+                    const int item = lq * kGroup + lgrp;
+                    uint32_t* bdst = &sm.bmring[warp][d][lane];
                     if (item < nact) {
                         const unsigned jj = sm.ent[item] >> 16;
                         const uint32_t ci = sm.colinfo[jj];
-                        bytes = (((ci & 0xFFFFu) + 7u) & ~7u) * 2u;
-                        src = p.values + (static_cast<uint64_t>(sm.tileoff[jj >> 4]) + (ci >> 16));
-                    }
-                    unsigned total = bytes + __shfl_xor_sync(0xFFFFFFFFu, bytes, 1);
-                    total += __shfl_xor_sync(0xFFFFFFFFu, total, 2);
-                    if (lq < ngroups) {
-                        mbar_wait(smem_u32(&sm.empty[s]), (use & 1u) ^ 1u, abort_flag, p.status);
-                        const uint32_t fb = smem_u32(&sm.full[s]);
-                        if ((lane & 3) == 0) mbar_arrive_expect_tx(fb, total);
-                        if (bytes != 0)
-                            bulk_g2s(ring_base + s * kStageBytes + (lane & 3) * kSlotBytes, src, bytes, fb);
+                        const int nch = static_cast<int>(((ci & 0xFFFFu) + 7u) >> 3);       // 16-byte pieces
+                        const unsigned char* src = val8 + 2 * (static_cast<uint64_t>(sm.tileoff[jj >> 4]) + (ci >> 16))
+                                                   + 16 * (lane & 7);
+                        const uint32_t dst = smem_u32(&sm.ring[warp][d][lgrp * kSlotBytes + 16 * (lane & 7)]);
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            cp_async16(dst + 128 * k, src + 128 * k, (lane & 7) + 8 * k < nch);
+                        cp_async4(smem_u32(bdst), bm8 + (row_slot0 + j0 + jj) * 32 + (lane & 7) * 4);
+                    } else {
+                        *bdst = 0u;
                     }
                 }
-            } else {
-                // ---- (2b) consumer warp: groups G with G % kConsumers == warp ----
-                const int lq0 = static_cast<int>((warp + kConsumers - gbase % kConsumers) % kConsumers);
-                const unsigned char* bm8 = reinterpret_cast<const unsigned char*>(p.bitmap);
-                auto prefetch_bitmaps = [&](int lq) {
-                    if (lq < ngroups) {
-                        const unsigned G = gbase + lq;
-                        const unsigned d = (G % kStages) / kConsumers;
-                        const int item = lq * kGroup + (lane >> 3);
-                        uint32_t* dst = &sm.bmring[warp][d][lane];
-                        if (item < nact) {
-                            const int64_t slot = row_slot0 + j0 + (sm.ent[item] >> 16);
-                            cp_async4(smem_u32(dst), bm8 + slot * 32 + (lane & 7) * 4);
-                        } else {
-                            *dst = 0u;
-                        }
-                    }
-                    cp_async_commit();
-                };
+                cp_async_commit();
+            };
 #pragma unroll
-                for (int d = 0; d < kDepth; ++d) prefetch_bitmaps(lq0 + d * kConsumers);
+            for (int d = 0; d < kDepth; ++d) fetch(d);
 
-                for (int lq = lq0; lq < ngroups; lq += kConsumers) {
-                    const unsigned G = gbase + lq;
-                    const unsigned s = G % kStages, use = G / kStages;
-                    cp_async_wait<kDepth - 1>();
-                    __syncwarp();
-                    const unsigned myword = sm.bmring[warp][s / kConsumers][lane];   // word (lane&7) of item lane>>3
-                    // exclusive prefix of the word popcounts inside each column tile (8-lane segments)
-                    const unsigned cnt = __popc(myword);
-                    unsigned inc = cnt;
+            for (int i = 0; warp + i * kWarps < ngroups; ++i) {
+                const int lq = warp + i * kWarps;
+                const int d = i % kDepth;
+                cp_async_wait<kDepth - 1>();
+                __syncwarp();
+                const unsigned myword = sm.bmring[warp][d][lane];       // word (lane&7) of item lane>>3
+                // exclusive prefix of the word popcounts inside each column tile (8-lane segments)
+                const unsigned cnt = __popc(myword);
+                unsigned inc = cnt;
 #pragma unroll
-                    for (int d = 1; d < 8; d <<= 1) {
-                        unsigned v = __shfl_up_sync(0xFFFFFFFFu, inc, d, 8);
-                        if ((lane & 7) >= d) inc += v;
-                    }
-                    const unsigned excl = inc - cnt;
-                    mbar_wait(smem_u32(&sm.full[s]), use & 1u, abort_flag, p.status);
-                    const uint32_t stage_base = ring_base + s * kStageBytes;
-#pragma unroll
-                    for (int it = 0; it < kGroup; ++it) {
-                        const int item = lq * kGroup + it;
-                        const unsigned short xh = static_cast<unsigned short>(sm.ent[item < nact ? item : 0] & 0xFFFFu);
-#pragma unroll
-                        for (int h = 0; h < 2; ++h) {
-                            const int src_lane = it * 8 + h * 4 + lgrp;
-                            const unsigned W = __shfl_sync(0xFFFFFFFFu, myword, src_lane);
-                            const unsigned E = __shfl_sync(0xFFFFFFFFu, excl, src_lane);
-                            const unsigned rank = E + __popc(W & lt_mask);
-                            const unsigned nib = W >> sh;
-                            uint32_t a = stage_base + it * kSlotBytes + 2u * rank;
-                            if (nib & 1u) { fma_f16(acc[4 * h + 0], lds_u16(a), xh); a += 2; }
-                            if (nib & 2u) { fma_f16(acc[4 * h + 1], lds_u16(a), xh); a += 2; }
-                            if (nib & 4u) { fma_f16(acc[4 * h + 2], lds_u16(a), xh); a += 2; }
-                            if (nib & 8u) { fma_f16(acc[4 * h + 3], lds_u16(a), xh); }
-                        }
-                    }
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&sm.empty[s]));
-                    prefetch_bitmaps(lq + kDepth * kConsumers);
+                for (int dd = 1; dd < 8; dd <<= 1) {
+                    unsigned v = __shfl_up_sync(0xFFFFFFFFu, inc, dd, 8);
+                    if ((lane & 7) >= dd) inc += v;
                 }
-                cp_async_wait<0>();
+                const unsigned excl = inc - cnt;
+                const unsigned char* stage = &sm.ring[warp][d][0];
+#pragma unroll
+                for (int it = 0; it < kGroup; ++it) {
+                    const int item = lq * kGroup + it;
+                    const unsigned short xh = static_cast<unsigned short>(sm.ent[item < nact ? item : 0] & 0xFFFFu);
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const int src_lane = it * 8 + h * 4 + lgrp;
+                        const unsigned W = __shfl_sync(0xFFFFFFFFu, myword, src_lane);
+                        const unsigned E = __shfl_sync(0xFFFFFFFFu, excl, src_lane);
+                        const unsigned rank = E + __popc(W & lt_mask);
+                        const unsigned nib = W >> sh;
+                        const unsigned short* v = reinterpret_cast<const unsigned short*>(stage + it * kSlotBytes) + rank;
+                        if (nib & 1u) { fma_f16(acc[4 * h + 0], *v, xh); ++v; }
+                        if (nib & 2u) { fma_f16(acc[4 * h + 1], *v, xh); ++v; }
+                        if (nib & 4u) { fma_f16(acc[4 * h + 2], *v, xh); ++v; }
+                        if (nib & 8u) { fma_f16(acc[4 * h + 3], *v, xh); }
+                    }
+                }
+                __syncwarp();                  // everyone is done with ring position d
+                fetch(i + kDepth);
             }
-            gbase += static_cast<unsigned>(ngroups);
+            cp_async_wait<0>();
             __syncthreads();       // the chunk's shared tables are rebuilt next
         }
 
-        // ---- (3) row reduction across the consumer warps (fixed order) ----
-        if (!is_producer) {
+        // ---- (3) row reduction across the warps (fixed order) ----
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                sm.red[warp][4 * lane + k] = acc[k];
-                sm.red[warp][128 + 4 * lane + k] = acc[4 + k];
-            }
+        for (int k = 0; k < 4; ++k) {
+            sm.red[warp][4 * lane + k] = acc[k];
+            sm.red[warp][128 + 4 * lane + k] = acc[4 + k];
         }
         __syncthreads();
         float part = 0.f;
         const int64_t row = static_cast<int64_t>(r) * kTileM + t;
         if (t < kTileM) {
 #pragma unroll
-            for (int w = 0; w < kConsumers; ++w) part += sm.red[w][t];
+            for (int w = 0; w < kWarps; ++w) part += sm.red[w][t];
         }
         // ---- split-K combine ----
         const int nseg = p.row_nseg[r];

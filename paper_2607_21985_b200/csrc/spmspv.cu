@@ -51,7 +51,7 @@ struct __align__(128) Smem {
     uint32_t bmring[kWarps][kDepth][32];                // their bitmap words (8 words x 4 column tiles)
     uint32_t colinfo[kChunkCols];                       // ColInfo words of the chunk's GTiles
     uint32_t tileoff[kChunkGT + 1];                     // TileOffset of the chunk's GTiles
-    uint32_t ent[kChunkCols];                           // active list: (column in chunk) << 16 | x bits
+    uint32_t ent[kChunkCols + kGroup];                  // active list: (column in chunk) << 16 | x bits
     float red[kWarps][kTileM];
     uint32_t group_mask[kChunkCols / 32];
     uint32_t group_base[kChunkCols / 32 + 1];
@@ -85,9 +85,49 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-// acc += w * x with fp16 operands and an fp32 accumulator: the product of two fp16 is exact in fp32.
-__device__ __forceinline__ void fma_f16(float& acc, unsigned short w, unsigned short x) {
-    asm("fma.rn.f32.f16 %0, %1, %2, %0;" : "+f"(acc) : "h"(w), "h"(x));
+// One decode step (Sec. 4.2.1): the 4 consecutive rows this lane owns inside the 32-bit bitmap
+// word W.  A is the shared-memory address of the word's first value, below the bits of lower
+// nibbles, m0..m3 the lane's four bits.  rank = set bits before the position; a set bit takes the
+// next value and adds value * x to its row's fp32 accumulator.  fma.rn.f32.f16 multiplies two fp16
+// exactly and accumulates in fp32.
+__device__ __forceinline__ void decode_step(unsigned W, uint32_t A, unsigned below, unsigned m0, unsigned m1,
+                                            unsigned m2, unsigned m3, unsigned x32, float& a0, float& a1,
+                                            float& a2, float& a3) {
+    asm volatile(
+        "{\n"
+        " .reg .pred p0, p1, p2, p3;\n"
+        " .reg .b16 v0, v1, v2, v3, xl, xu;\n"
+        " .reg .b32 t, a;\n"
+        " and.b32 t, %4, %6;\n"
+        " popc.b32 t, t;\n"
+        " shl.b32 t, t, 1;\n"
+        " add.u32 a, %5, t;\n"
+        " and.b32 t, %4, %7;\n setp.ne.u32 p0, t, 0;\n"
+        " and.b32 t, %4, %8;\n setp.ne.u32 p1, t, 0;\n"
+        " and.b32 t, %4, %9;\n setp.ne.u32 p2, t, 0;\n"
+        " and.b32 t, %4, %10;\n setp.ne.u32 p3, t, 0;\n"
+        " mov.b32 {xl, xu}, %11;\n"
+        " @p0 ld.shared.u16 v0, [a];\n @p0 add.u32 a, a, 2;\n"
+        " @p1 ld.shared.u16 v1, [a];\n @p1 add.u32 a, a, 2;\n"
+        " @p2 ld.shared.u16 v2, [a];\n @p2 add.u32 a, a, 2;\n"
+        " @p3 ld.shared.u16 v3, [a];\n"
+        " @p0 fma.rn.f32.f16 %0, v0, xl, %0;\n"
+        " @p1 fma.rn.f32.f16 %1, v1, xl, %1;\n"
+        " @p2 fma.rn.f32.f16 %2, v2, xl, %2;\n"
+        " @p3 fma.rn.f32.f16 %3, v3, xl, %3;\n"
+        "}"
+        : "+f"(a0), "+f"(a1), "+f"(a2), "+f"(a3)
+        : "r"(W), "r"(A), "r"(below), "r"(m0), "r"(m1), "r"(m2), "r"(m3), "r"(x32));
+}
+__device__ __forceinline__ unsigned lds_u16(uint32_t addr) {
+    unsigned v;
+    asm volatile("{\n .reg .b16 h;\n ld.shared.u16 h, [%1];\n cvt.u32.u16 %0, h;\n}" : "=r"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ unsigned lds_u32(uint32_t addr) {
+    unsigned v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
 }
 
 // One persistent CTA per GTile range; every warp runs its own fetch -> decode pipeline.
@@ -110,9 +150,14 @@ spmspv_kernel(const Params p) {
     const int64_t g_begin = p.cta_begin[blockIdx.x], g_end = p.cta_begin[blockIdx.x + 1];
     const int r_first = static_cast<int>(g_begin / p.C);
 
-    const unsigned sh = 4u * (lane & 7);            // my nibble inside a 32-bit bitmap word
-    const unsigned lt_mask = (1u << sh) - 1u;
+    const int lane7 = lane & 7;
     const int lgrp = lane >> 3;                     // which item of a group I fetch for / which word I decode
+    const unsigned bit0 = 1u << (4 * lane7);        // first bit of my nibble inside a 32-bit bitmap word
+    const unsigned lt_mask = bit0 - 1u;
+    const uint32_t val_ring = smem_u32(&sm.ring[warp][0][lgrp * kSlotBytes + 16 * lane7]);   // my fetch destination
+    const uint32_t val_slot = smem_u32(&sm.ring[warp][0][lgrp * kSlotBytes]);                // my word's column tile
+    const uint32_t bm_ring = smem_u32(&sm.bmring[warp][0][lane]);
+    const uint32_t ent_addr = smem_u32(&sm.ent[0]);
     const unsigned char* bm8 = reinterpret_cast<const unsigned char*>(p.bitmap);
     const unsigned char* val8 = reinterpret_cast<const unsigned char*>(p.values);
 
@@ -176,26 +221,27 @@ spmspv_kernel(const Params p) {
             const int ngroups = (nact + kGroup - 1) / kGroup;
 
             // ---- (2) per-warp fetch / decode pipeline over groups warp, warp + kWarps, ... ----
-            // fetch(i): start the copies of my i-th group into ring position i % kDepth
+            const unsigned char* bm_chunk = bm8 + (row_slot0 + j0) * 32 + lane7 * 4;
+            // fetch(i): start the copies of my i-th group into ring position i % kDepth.  Lane
+            // (lgrp, lane7) moves pieces lane7, lane7+8, ... of the group's lgrp-th column tile.
             auto fetch = [&](int i) {
                 const int lq = warp + i * kWarps;
                 if (lq < ngroups) {
                     const int d = i % kDepth;
                     const int item = lq * kGroup + lgrp;
-                    uint32_t* bdst = &sm.bmring[warp][d][lane];
+                    const uint32_t bdst = bm_ring + d * 128;
                     if (item < nact) {
                         const unsigned jj = sm.ent[item] >> 16;
                         const uint32_t ci = sm.colinfo[jj];
-                        const int nch = static_cast<int>(((ci & 0xFFFFu) + 7u) >> 3);       // 16-byte pieces
+                        const int rem = static_cast<int>(((ci & 0xFFFFu) + 7u) >> 3) - lane7;   // my 16-byte pieces left
                         const unsigned char* src = val8 + 2 * (static_cast<uint64_t>(sm.tileoff[jj >> 4]) + (ci >> 16))
-                                                   + 16 * (lane & 7);
-                        const uint32_t dst = smem_u32(&sm.ring[warp][d][lgrp * kSlotBytes + 16 * (lane & 7)]);
+                                                   + 16 * lane7;
+                        const uint32_t dst = val_ring + d * kStageBytes;
 #pragma unroll
-                        for (int k = 0; k < 4; ++k)
-                            cp_async16(dst + 128 * k, src + 128 * k, (lane & 7) + 8 * k < nch);
-                        cp_async4(smem_u32(bdst), bm8 + (row_slot0 + j0 + jj) * 32 + (lane & 7) * 4);
+                        for (int k = 0; k < 4; ++k) cp_async16(dst + 128 * k, src + 128 * k, rem > 8 * k);
+                        cp_async4(bdst, bm_chunk + static_cast<size_t>(jj) * 32);
                     } else {
-                        *bdst = 0u;
+                        asm volatile("st.shared.u32 [%0], %1;" ::"r"(bdst), "r"(0u) : "memory");
                     }
                 }
                 cp_async_commit();
@@ -203,42 +249,36 @@ spmspv_kernel(const Params p) {
 #pragma unroll
             for (int d = 0; d < kDepth; ++d) fetch(d);
 
-            for (int i = 0; warp + i * kWarps < ngroups; ++i) {
-                const int lq = warp + i * kWarps;
-                const int d = i % kDepth;
+            int d = 0;
+            for (int i = 0, lq = warp; lq < ngroups; ++i, lq += kWarps) {
                 cp_async_wait<kDepth - 1>();
                 __syncwarp();
-                const unsigned myword = sm.bmring[warp][d][lane];       // word (lane&7) of item lane>>3
-                // exclusive prefix of the word popcounts inside each column tile (8-lane segments)
+                // my word: word lane7 of the group's lgrp-th column tile; A = address of its first value
+                const unsigned myword = lds_u32(bm_ring + d * 128);
                 const unsigned cnt = __popc(myword);
                 unsigned inc = cnt;
 #pragma unroll
                 for (int dd = 1; dd < 8; dd <<= 1) {
                     unsigned v = __shfl_up_sync(0xFFFFFFFFu, inc, dd, 8);
-                    if ((lane & 7) >= dd) inc += v;
+                    if (lane7 >= dd) inc += v;
                 }
-                const unsigned excl = inc - cnt;
-                const unsigned char* stage = &sm.ring[warp][d][0];
+                const uint32_t myA = val_slot + d * kStageBytes + 2u * (inc - cnt);
+                const uint32_t xaddr = ent_addr + 4u * (lq * kGroup);
 #pragma unroll
                 for (int it = 0; it < kGroup; ++it) {
-                    const int item = lq * kGroup + it;
-                    const unsigned short xh = static_cast<unsigned short>(sm.ent[item < nact ? item : 0] & 0xFFFFu);
+                    const unsigned x32 = lds_u16(xaddr + 4 * it);          // x bits of the it-th column (low half of ent)
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
                         const int src_lane = it * 8 + h * 4 + lgrp;
                         const unsigned W = __shfl_sync(0xFFFFFFFFu, myword, src_lane);
-                        const unsigned E = __shfl_sync(0xFFFFFFFFu, excl, src_lane);
-                        const unsigned rank = E + __popc(W & lt_mask);
-                        const unsigned nib = W >> sh;
-                        const unsigned short* v = reinterpret_cast<const unsigned short*>(stage + it * kSlotBytes) + rank;
-                        if (nib & 1u) { fma_f16(acc[4 * h + 0], *v, xh); ++v; }
-                        if (nib & 2u) { fma_f16(acc[4 * h + 1], *v, xh); ++v; }
-                        if (nib & 4u) { fma_f16(acc[4 * h + 2], *v, xh); ++v; }
-                        if (nib & 8u) { fma_f16(acc[4 * h + 3], *v, xh); }
+                        const uint32_t A = __shfl_sync(0xFFFFFFFFu, myA, src_lane);
+                        decode_step(W, A, lt_mask, bit0, bit0 << 1, bit0 << 2, bit0 << 3, x32,
+                                    acc[4 * h + 0], acc[4 * h + 1], acc[4 * h + 2], acc[4 * h + 3]);
                     }
                 }
                 __syncwarp();                  // everyone is done with ring position d
                 fetch(i + kDepth);
+                d = (d + 1 == kDepth) ? 0 : d + 1;
             }
             cp_async_wait<0>();
             __syncthreads();       // the chunk's shared tables are rebuilt next

@@ -10,6 +10,7 @@
 // another, and the order of the additions is fixed.  Only the first and the last segment of a
 // CTA can share their row tile with another CTA, so a CTA owns two workspace slots: slot 0 for
 // the row tile its range starts in, slot 1 for any later one.
+#include <cstddef>
 #include <mutex>
 
 #include "spdp_internal.h"
@@ -17,10 +18,17 @@
 namespace spdp {
 namespace {
 
-constexpr int kWarps = 16;                 // warps per CTA; every warp fetches and decodes its own column tiles
-constexpr int kDepth = 3;                  // groups a warp keeps in flight
+#ifndef SPDP_WARPS
+#define SPDP_WARPS 24
+#endif
+#ifndef SPDP_DEPTH
+#define SPDP_DEPTH 2
+#endif
+constexpr int kWarps = SPDP_WARPS;         // warps per CTA; every warp fetches and decodes its own column tiles
+constexpr int kDepth = SPDP_DEPTH;         // groups a warp keeps in flight
 constexpr int kGroup = 4;                  // active column tiles per group (one fetch / decode unit of a warp)
-constexpr int kSlotBytes = 2 * kTileM;     // a column tile's values: at most 256 fp16
+constexpr int kSlotBytes = 2 * kTileM + 32;  // a column tile's values (at most 256 fp16) + 32 bytes so that the
+                                             // four tiles of a group start 8 banks apart
 constexpr int kStageBytes = kGroup * kSlotBytes;
 constexpr int kThreads = kWarps * 32;
 constexpr int kChunkCols = 8192;           // columns handled between two pipeline drains
@@ -47,16 +55,24 @@ struct Params {
 };
 
 struct __align__(128) Smem {
-    unsigned char ring[kWarps][kDepth][kStageBytes];    // values of the column tiles in flight, per warp
-    uint32_t bmring[kWarps][kDepth][32];                // their bitmap words (8 words x 4 column tiles)
+    union {
+        unsigned char ring[kWarps][kDepth][kStageBytes];    // values of the column tiles in flight, per warp
+        float red[kWarps][kTileM];                          // cross-warp row reduction (after the pipelines drained)
+    };
+    // Bitmap words of a group in decode order: word w of the group's it-th tile sits at
+    // [(w & 3) * 8 + it * 2 + (w >> 2)], so the lanes that decode words (w & 3) == g read 8 consecutive words.
+    alignas(16) uint32_t bmring[kWarps][kDepth][32];
+    alignas(16) unsigned short voff[kWarps][32];                    // same order: byte offset of each word's first value in its slot
     uint32_t colinfo[kChunkCols];                       // ColInfo words of the chunk's GTiles
     uint32_t tileoff[kChunkGT + 1];                     // TileOffset of the chunk's GTiles
-    uint32_t ent[kChunkCols + kGroup];                  // active list: (column in chunk) << 16 | x bits
-    float red[kWarps][kTileM];
+    alignas(16) uint32_t ent[kChunkCols + kGroup];      // active list: (column in chunk) << 16 | x bits (read 4 at a time)
     uint32_t group_mask[kChunkCols / 32];
     uint32_t group_base[kChunkCols / 32 + 1];
     int is_last;
 };
+static_assert(offsetof(Smem, ent) % 16 == 0 && offsetof(Smem, voff) % 16 == 0 && offsetof(Smem, bmring) % 16 == 0,
+              "16-byte shared loads need aligned tables");
+static_assert(sizeof(float) * kWarps * kTileM <= size_t(kWarps) * kDepth * kStageBytes, "red must fit in the ring");
 
 // DP test of Sec. 4.2 step (3): magnitude against the threshold; NOT(|x| <= thr) keeps NaN.
 __device__ __forceinline__ bool column_active(int rule, float thr, const uint32_t* mask, int j, __half xj) {
@@ -86,11 +102,12 @@ template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 // One decode step (Sec. 4.2.1): the 4 consecutive rows this lane owns inside the 32-bit bitmap
-// word W.  A is the shared-memory address of the word's first value, below the bits of lower
-// nibbles, m0..m3 the lane's four bits.  rank = set bits before the position; a set bit takes the
-// next value and adds value * x to its row's fp32 accumulator.  fma.rn.f32.f16 multiplies two fp16
-// exactly and accumulates in fp32.
-__device__ __forceinline__ void decode_step(unsigned W, uint32_t A, unsigned below, unsigned m0, unsigned m1,
+// word W.  `first` is the shared-memory address of the word's first value (kOff is added to every
+// access), `below` masks the bits of lower nibbles, m0..m3 are the lane's four bits.
+// rank = set bits before the position; a set bit takes the next value and adds value * x to its
+// row's fp32 accumulator.  fma.rn.f32.f16 multiplies two fp16 exactly and accumulates in fp32.
+template <int kOff>
+__device__ __forceinline__ void decode_step(unsigned W, uint32_t first, unsigned below, unsigned m0, unsigned m1,
                                             unsigned m2, unsigned m3, unsigned x32, float& a0, float& a1,
                                             float& a2, float& a3) {
     asm volatile(
@@ -107,27 +124,33 @@ __device__ __forceinline__ void decode_step(unsigned W, uint32_t A, unsigned bel
         " and.b32 t, %4, %9;\n setp.ne.u32 p2, t, 0;\n"
         " and.b32 t, %4, %10;\n setp.ne.u32 p3, t, 0;\n"
         " mov.b32 {xl, xu}, %11;\n"
-        " @p0 ld.shared.u16 v0, [a];\n @p0 add.u32 a, a, 2;\n"
-        " @p1 ld.shared.u16 v1, [a];\n @p1 add.u32 a, a, 2;\n"
-        " @p2 ld.shared.u16 v2, [a];\n @p2 add.u32 a, a, 2;\n"
-        " @p3 ld.shared.u16 v3, [a];\n"
+        " @p0 ld.shared.u16 v0, [a+%12];\n @p0 add.u32 a, a, 2;\n"
+        " @p1 ld.shared.u16 v1, [a+%12];\n @p1 add.u32 a, a, 2;\n"
+        " @p2 ld.shared.u16 v2, [a+%12];\n @p2 add.u32 a, a, 2;\n"
+        " @p3 ld.shared.u16 v3, [a+%12];\n"
         " @p0 fma.rn.f32.f16 %0, v0, xl, %0;\n"
         " @p1 fma.rn.f32.f16 %1, v1, xl, %1;\n"
         " @p2 fma.rn.f32.f16 %2, v2, xl, %2;\n"
         " @p3 fma.rn.f32.f16 %3, v3, xl, %3;\n"
         "}"
         : "+f"(a0), "+f"(a1), "+f"(a2), "+f"(a3)
-        : "r"(W), "r"(A), "r"(below), "r"(m0), "r"(m1), "r"(m2), "r"(m3), "r"(x32));
-}
-__device__ __forceinline__ unsigned lds_u16(uint32_t addr) {
-    unsigned v;
-    asm volatile("{\n .reg .b16 h;\n ld.shared.u16 h, [%1];\n cvt.u32.u16 %0, h;\n}" : "=r"(v) : "r"(addr));
-    return v;
+        : "r"(W), "r"(first), "r"(below), "r"(m0), "r"(m1), "r"(m2), "r"(m3), "r"(x32), "n"(kOff));
 }
 __device__ __forceinline__ unsigned lds_u32(uint32_t addr) {
     unsigned v;
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
     return v;
+}
+__device__ __forceinline__ uint4 lds_v4(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ void sts_u16(uint32_t addr, unsigned v) {
+    asm volatile("{\n .reg .b16 h;\n cvt.u16.u32 h, %1;\n st.shared.u16 [%0], h;\n}" ::"r"(addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ void sts_u32(uint32_t addr, unsigned v) {
+    asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
 
 // One persistent CTA per GTile range; every warp runs its own fetch -> decode pipeline.
@@ -151,12 +174,19 @@ spmspv_kernel(const Params p) {
     const int r_first = static_cast<int>(g_begin / p.C);
 
     const int lane7 = lane & 7;
-    const int lgrp = lane >> 3;                     // which item of a group I fetch for / which word I decode
+    const int lgrp = lane >> 3;
     const unsigned bit0 = 1u << (4 * lane7);        // first bit of my nibble inside a 32-bit bitmap word
     const unsigned lt_mask = bit0 - 1u;
-    const uint32_t val_ring = smem_u32(&sm.ring[warp][0][lgrp * kSlotBytes + 16 * lane7]);   // my fetch destination
-    const uint32_t val_slot = smem_u32(&sm.ring[warp][0][lgrp * kSlotBytes]);                // my word's column tile
-    const uint32_t bm_ring = smem_u32(&sm.bmring[warp][0][lane]);
+    // fetch role: lane (lgrp, lane7) moves 16-byte pieces lane7, lane7+8, ... and bitmap word lane7 of the
+    // group's lgrp-th tile.  scan role: the same (tile, word).  decode role: nibble lane7 of words w with
+    // (w & 3) == lgrp of every tile of the group.
+    const int tpos = (lane7 & 3) * 8 + lgrp * 2 + (lane7 >> 2);         // where (tile lgrp, word lane7) sits
+    const uint32_t val_dst = smem_u32(&sm.ring[warp][0][lgrp * kSlotBytes + 16 * lane7]);
+    const uint32_t val_base = smem_u32(&sm.ring[warp][0][0]);
+    const uint32_t bm_own = smem_u32(&sm.bmring[warp][0][tpos]);
+    const uint32_t bm_dec = smem_u32(&sm.bmring[warp][0][lgrp * 8]);
+    const uint32_t voff_own = smem_u32(&sm.voff[warp][tpos]);
+    const uint32_t voff_dec = smem_u32(&sm.voff[warp][lgrp * 8]);
     const uint32_t ent_addr = smem_u32(&sm.ent[0]);
     const unsigned char* bm8 = reinterpret_cast<const unsigned char*>(p.bitmap);
     const unsigned char* val8 = reinterpret_cast<const unsigned char*>(p.values);
@@ -222,26 +252,25 @@ spmspv_kernel(const Params p) {
 
             // ---- (2) per-warp fetch / decode pipeline over groups warp, warp + kWarps, ... ----
             const unsigned char* bm_chunk = bm8 + (row_slot0 + j0) * 32 + lane7 * 4;
-            // fetch(i): start the copies of my i-th group into ring position i % kDepth.  Lane
-            // (lgrp, lane7) moves pieces lane7, lane7+8, ... of the group's lgrp-th column tile.
+            // fetch(i): start the copies of my i-th group into ring position i % kDepth
             auto fetch = [&](int i) {
                 const int lq = warp + i * kWarps;
                 if (lq < ngroups) {
                     const int d = i % kDepth;
                     const int item = lq * kGroup + lgrp;
-                    const uint32_t bdst = bm_ring + d * 128;
+                    const uint32_t bdst = bm_own + d * 128;
                     if (item < nact) {
                         const unsigned jj = sm.ent[item] >> 16;
                         const uint32_t ci = sm.colinfo[jj];
                         const int rem = static_cast<int>(((ci & 0xFFFFu) + 7u) >> 3) - lane7;   // my 16-byte pieces left
                         const unsigned char* src = val8 + 2 * (static_cast<uint64_t>(sm.tileoff[jj >> 4]) + (ci >> 16))
                                                    + 16 * lane7;
-                        const uint32_t dst = val_ring + d * kStageBytes;
+                        const uint32_t dst = val_dst + d * kStageBytes;
 #pragma unroll
                         for (int k = 0; k < 4; ++k) cp_async16(dst + 128 * k, src + 128 * k, rem > 8 * k);
                         cp_async4(bdst, bm_chunk + static_cast<size_t>(jj) * 32);
                     } else {
-                        asm volatile("st.shared.u32 [%0], %1;" ::"r"(bdst), "r"(0u) : "memory");
+                        sts_u32(bdst, 0u);
                     }
                 }
                 cp_async_commit();
@@ -253,38 +282,41 @@ spmspv_kernel(const Params p) {
             for (int i = 0, lq = warp; lq < ngroups; ++i, lq += kWarps) {
                 cp_async_wait<kDepth - 1>();
                 __syncwarp();
-                // my word: word lane7 of the group's lgrp-th column tile; A = address of its first value
-                const unsigned myword = lds_u32(bm_ring + d * 128);
-                const unsigned cnt = __popc(myword);
-                unsigned inc = cnt;
+                // scan role: byte offset of my word's first value inside its tile's slot
+                {
+                    const unsigned cnt = __popc(lds_u32(bm_own + d * 128));
+                    unsigned inc = cnt;
 #pragma unroll
-                for (int dd = 1; dd < 8; dd <<= 1) {
-                    unsigned v = __shfl_up_sync(0xFFFFFFFFu, inc, dd, 8);
-                    if (lane7 >= dd) inc += v;
-                }
-                const uint32_t myA = val_slot + d * kStageBytes + 2u * (inc - cnt);
-                const uint32_t xaddr = ent_addr + 4u * (lq * kGroup);
-#pragma unroll
-                for (int it = 0; it < kGroup; ++it) {
-                    const unsigned x32 = lds_u16(xaddr + 4 * it);          // x bits of the it-th column (low half of ent)
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        const int src_lane = it * 8 + h * 4 + lgrp;
-                        const unsigned W = __shfl_sync(0xFFFFFFFFu, myword, src_lane);
-                        const uint32_t A = __shfl_sync(0xFFFFFFFFu, myA, src_lane);
-                        decode_step(W, A, lt_mask, bit0, bit0 << 1, bit0 << 2, bit0 << 3, x32,
-                                    acc[4 * h + 0], acc[4 * h + 1], acc[4 * h + 2], acc[4 * h + 3]);
+                    for (int dd = 1; dd < 8; dd <<= 1) {
+                        unsigned v = __shfl_up_sync(0xFFFFFFFFu, inc, dd, 8);
+                        if (lane7 >= dd) inc += v;
                     }
+                    sts_u16(voff_own, 2u * (inc - cnt));
                 }
+                __syncwarp();
+                // decode role: my 8 words (tile it, word 4h + lgrp at index 2*it + h), their offsets, the 4 x
+                const uint4 w03 = lds_v4(bm_dec + d * 128), w47 = lds_v4(bm_dec + d * 128 + 16);
+                const uint4 off = lds_v4(voff_dec);
+                const uint4 xs = lds_v4(ent_addr + 16u * lq);
+                const uint32_t stage = val_base + d * kStageBytes;
+                const unsigned m1 = bit0 << 1, m2 = bit0 << 2, m3 = bit0 << 3;
+                decode_step<0 * kSlotBytes>(w03.x, stage + (off.x & 0xFFFFu), lt_mask, bit0, m1, m2, m3, xs.x, acc[0], acc[1], acc[2], acc[3]);
+                decode_step<0 * kSlotBytes>(w03.y, stage + (off.x >> 16), lt_mask, bit0, m1, m2, m3, xs.x, acc[4], acc[5], acc[6], acc[7]);
+                decode_step<1 * kSlotBytes>(w03.z, stage + (off.y & 0xFFFFu), lt_mask, bit0, m1, m2, m3, xs.y, acc[0], acc[1], acc[2], acc[3]);
+                decode_step<1 * kSlotBytes>(w03.w, stage + (off.y >> 16), lt_mask, bit0, m1, m2, m3, xs.y, acc[4], acc[5], acc[6], acc[7]);
+                decode_step<2 * kSlotBytes>(w47.x, stage + (off.z & 0xFFFFu), lt_mask, bit0, m1, m2, m3, xs.z, acc[0], acc[1], acc[2], acc[3]);
+                decode_step<2 * kSlotBytes>(w47.y, stage + (off.z >> 16), lt_mask, bit0, m1, m2, m3, xs.z, acc[4], acc[5], acc[6], acc[7]);
+                decode_step<3 * kSlotBytes>(w47.z, stage + (off.w & 0xFFFFu), lt_mask, bit0, m1, m2, m3, xs.w, acc[0], acc[1], acc[2], acc[3]);
+                decode_step<3 * kSlotBytes>(w47.w, stage + (off.w >> 16), lt_mask, bit0, m1, m2, m3, xs.w, acc[4], acc[5], acc[6], acc[7]);
                 __syncwarp();                  // everyone is done with ring position d
                 fetch(i + kDepth);
                 d = (d + 1 == kDepth) ? 0 : d + 1;
             }
             cp_async_wait<0>();
-            __syncthreads();       // the chunk's shared tables are rebuilt next
+            __syncthreads();       // the chunk's shared tables are rebuilt next; the ring is idle
         }
 
-        // ---- (3) row reduction across the warps (fixed order) ----
+        // ---- (3) row reduction across the warps (fixed order); red[] reuses the idle ring ----
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
             sm.red[warp][4 * lane + k] = acc[k];
@@ -326,7 +358,7 @@ spmspv_kernel(const Params p) {
                 if (t == 0) p.row_counter[r] = 0;       // ready for the next call on this handle
             }
         }
-        __syncthreads();           // red[] and is_last are reused by the next segment
+        __syncthreads();           // red[] (the ring) and is_last are reused by the next segment
     }
 }
 

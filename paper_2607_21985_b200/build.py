@@ -35,6 +35,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     flags = [f for f in NVCC_FLAGS if not f.startswith("--use_fast_math")]
     if verbose:
         flags += ["-Xptxas", "-v"]
+    flags += os.environ.get("SPDP_NVCC_EXTRA", "").split()      # tuning hook, e.g. -DSPDP_WARPS=20
     tmp = LIB + f".tmp{os.getpid()}"
     cmd = [nvcc(), *flags, "-shared", "-I", os.path.join(ROOT, "include"), "-I", os.path.join(HERE, "csrc"),
            "-o", tmp, *SOURCES]

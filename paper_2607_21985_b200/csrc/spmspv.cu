@@ -62,7 +62,7 @@ struct __align__(128) Smem {
     // Bitmap words of a group in decode order: word w of the group's it-th tile sits at
     // [(w & 3) * 8 + it * 2 + (w >> 2)], so the lanes that decode words (w & 3) == g read 8 consecutive words.
     alignas(16) uint32_t bmring[kWarps][kDepth][32];
-    alignas(16) unsigned short voff[kWarps][32];                    // same order: byte offset of each word's first value in its slot
+    alignas(16) uint32_t vaddr[kWarps][32];             // same order: shared address of each word's first value
     uint32_t colinfo[kChunkCols];                       // ColInfo words of the chunk's GTiles
     uint32_t tileoff[kChunkGT + 1];                     // TileOffset of the chunk's GTiles
     alignas(16) uint32_t ent[kChunkCols + kGroup];      // active list: (column in chunk) << 16 | x bits (read 4 at a time)
@@ -70,7 +70,7 @@ struct __align__(128) Smem {
     uint32_t group_base[kChunkCols / 32 + 1];
     int is_last;
 };
-static_assert(offsetof(Smem, ent) % 16 == 0 && offsetof(Smem, voff) % 16 == 0 && offsetof(Smem, bmring) % 16 == 0,
+static_assert(offsetof(Smem, ent) % 16 == 0 && offsetof(Smem, vaddr) % 16 == 0 && offsetof(Smem, bmring) % 16 == 0,
               "16-byte shared loads need aligned tables");
 static_assert(sizeof(float) * kWarps * kTileM <= size_t(kWarps) * kDepth * kStageBytes, "red must fit in the ring");
 
@@ -90,9 +90,10 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
 // Asynchronous global -> shared copies (Sec. 4.2.3: 128-bit per thread); `on` = false copies nothing.
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool on) {
-    asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %2, 0;\n @p cp.async.cg.shared.global [%0], [%1], 16;\n}"
-                 ::"r"(dst), "l"(src), "r"(static_cast<int>(on)) : "memory");
+template <int kOff>
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int rem) {
+    asm volatile("{\n .reg .pred p;\n setp.gt.s32 p, %2, %3;\n @p cp.async.cg.shared.global [%0+%4], [%1+%4], 16;\n}"
+                 ::"r"(dst), "l"(src), "r"(rem), "n"(kOff / 16), "n"(kOff) : "memory");
 }
 __device__ __forceinline__ void cp_async4(uint32_t dst, const void* src) {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
@@ -102,11 +103,10 @@ template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 // One decode step (Sec. 4.2.1): the 4 consecutive rows this lane owns inside the 32-bit bitmap
-// word W.  `first` is the shared-memory address of the word's first value (kOff is added to every
-// access), `below` masks the bits of lower nibbles, m0..m3 are the lane's four bits.
-// rank = set bits before the position; a set bit takes the next value and adds value * x to its
-// row's fp32 accumulator.  fma.rn.f32.f16 multiplies two fp16 exactly and accumulates in fp32.
-template <int kOff>
+// word W.  `first` is the shared-memory address of the word's first value, `below` masks the bits
+// of lower nibbles, m0..m3 are the lane's four bits.  rank = set bits before the position; a set
+// bit takes the next value and adds value * x to its row's fp32 accumulator.  fma.rn.f32.f16
+// multiplies two fp16 exactly and accumulates in fp32.
 __device__ __forceinline__ void decode_step(unsigned W, uint32_t first, unsigned below, unsigned m0, unsigned m1,
                                             unsigned m2, unsigned m3, unsigned x32, float& a0, float& a1,
                                             float& a2, float& a3) {
@@ -119,22 +119,22 @@ __device__ __forceinline__ void decode_step(unsigned W, uint32_t first, unsigned
         " popc.b32 t, t;\n"
         " shl.b32 t, t, 1;\n"
         " add.u32 a, %5, t;\n"
-        " and.b32 t, %4, %7;\n setp.ne.u32 p0, t, 0;\n"
-        " and.b32 t, %4, %8;\n setp.ne.u32 p1, t, 0;\n"
-        " and.b32 t, %4, %9;\n setp.ne.u32 p2, t, 0;\n"
-        " and.b32 t, %4, %10;\n setp.ne.u32 p3, t, 0;\n"
+        " lop3.or.b32 t|p0, %4, %7, 0, 0xC0, 0;\n"
+        " lop3.or.b32 t|p1, %4, %8, 0, 0xC0, 0;\n"
+        " lop3.or.b32 t|p2, %4, %9, 0, 0xC0, 0;\n"
+        " lop3.or.b32 t|p3, %4, %10, 0, 0xC0, 0;\n"
         " mov.b32 {xl, xu}, %11;\n"
-        " @p0 ld.shared.u16 v0, [a+%12];\n @p0 add.u32 a, a, 2;\n"
-        " @p1 ld.shared.u16 v1, [a+%12];\n @p1 add.u32 a, a, 2;\n"
-        " @p2 ld.shared.u16 v2, [a+%12];\n @p2 add.u32 a, a, 2;\n"
-        " @p3 ld.shared.u16 v3, [a+%12];\n"
+        " @p0 ld.shared.u16 v0, [a];\n @p0 add.u32 a, a, 2;\n"
+        " @p1 ld.shared.u16 v1, [a];\n @p1 add.u32 a, a, 2;\n"
+        " @p2 ld.shared.u16 v2, [a];\n @p2 add.u32 a, a, 2;\n"
+        " @p3 ld.shared.u16 v3, [a];\n"
         " @p0 fma.rn.f32.f16 %0, v0, xl, %0;\n"
         " @p1 fma.rn.f32.f16 %1, v1, xl, %1;\n"
         " @p2 fma.rn.f32.f16 %2, v2, xl, %2;\n"
         " @p3 fma.rn.f32.f16 %3, v3, xl, %3;\n"
         "}"
         : "+f"(a0), "+f"(a1), "+f"(a2), "+f"(a3)
-        : "r"(W), "r"(first), "r"(below), "r"(m0), "r"(m1), "r"(m2), "r"(m3), "r"(x32), "n"(kOff));
+        : "r"(W), "r"(first), "r"(below), "r"(m0), "r"(m1), "r"(m2), "r"(m3), "r"(x32));
 }
 __device__ __forceinline__ unsigned lds_u32(uint32_t addr) {
     unsigned v;
@@ -146,8 +146,10 @@ __device__ __forceinline__ uint4 lds_v4(uint32_t addr) {
     asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
     return v;
 }
-__device__ __forceinline__ void sts_u16(uint32_t addr, unsigned v) {
-    asm volatile("{\n .reg .b16 h;\n cvt.u16.u32 h, %1;\n st.shared.u16 [%0], h;\n}" ::"r"(addr), "r"(v) : "memory");
+__device__ __forceinline__ uint2 lds_v2(uint32_t addr) {
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+    return v;
 }
 __device__ __forceinline__ void sts_u32(uint32_t addr, unsigned v) {
     asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
@@ -182,11 +184,11 @@ spmspv_kernel(const Params p) {
     // (w & 3) == lgrp of every tile of the group.
     const int tpos = (lane7 & 3) * 8 + lgrp * 2 + (lane7 >> 2);         // where (tile lgrp, word lane7) sits
     const uint32_t val_dst = smem_u32(&sm.ring[warp][0][lgrp * kSlotBytes + 16 * lane7]);
-    const uint32_t val_base = smem_u32(&sm.ring[warp][0][0]);
     const uint32_t bm_own = smem_u32(&sm.bmring[warp][0][tpos]);
     const uint32_t bm_dec = smem_u32(&sm.bmring[warp][0][lgrp * 8]);
-    const uint32_t voff_own = smem_u32(&sm.voff[warp][tpos]);
-    const uint32_t voff_dec = smem_u32(&sm.voff[warp][lgrp * 8]);
+    const uint32_t va_own = smem_u32(&sm.vaddr[warp][tpos]);
+    const uint32_t va_dec = smem_u32(&sm.vaddr[warp][lgrp * 8]);
+    const uint32_t slot_own = smem_u32(&sm.ring[warp][0][lgrp * kSlotBytes]);      // scan role: my tile's slot
     const uint32_t ent_addr = smem_u32(&sm.ent[0]);
     const unsigned char* bm8 = reinterpret_cast<const unsigned char*>(p.bitmap);
     const unsigned char* val8 = reinterpret_cast<const unsigned char*>(p.values);
@@ -266,8 +268,10 @@ spmspv_kernel(const Params p) {
                         const unsigned char* src = val8 + 2 * (static_cast<uint64_t>(sm.tileoff[jj >> 4]) + (ci >> 16))
                                                    + 16 * lane7;
                         const uint32_t dst = val_dst + d * kStageBytes;
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) cp_async16(dst + 128 * k, src + 128 * k, rem > 8 * k);
+                        cp_async16<0>(dst, src, rem);
+                        cp_async16<128>(dst, src, rem);
+                        cp_async16<256>(dst, src, rem);
+                        cp_async16<384>(dst, src, rem);
                         cp_async4(bdst, bm_chunk + static_cast<size_t>(jj) * 32);
                     } else {
                         sts_u32(bdst, 0u);
@@ -282,7 +286,7 @@ spmspv_kernel(const Params p) {
             for (int i = 0, lq = warp; lq < ngroups; ++i, lq += kWarps) {
                 cp_async_wait<kDepth - 1>();
                 __syncwarp();
-                // scan role: byte offset of my word's first value inside its tile's slot
+                // scan role: shared address of my word's first value
                 {
                     const unsigned cnt = __popc(lds_u32(bm_own + d * 128));
                     unsigned inc = cnt;
@@ -291,23 +295,21 @@ spmspv_kernel(const Params p) {
                         unsigned v = __shfl_up_sync(0xFFFFFFFFu, inc, dd, 8);
                         if (lane7 >= dd) inc += v;
                     }
-                    sts_u16(voff_own, 2u * (inc - cnt));
+                    sts_u32(va_own, slot_own + d * kStageBytes + 2u * (inc - cnt));
                 }
                 __syncwarp();
-                // decode role: my 8 words (tile it, word 4h + lgrp at index 2*it + h), their offsets, the 4 x
-                const uint4 w03 = lds_v4(bm_dec + d * 128), w47 = lds_v4(bm_dec + d * 128 + 16);
-                const uint4 off = lds_v4(voff_dec);
-                const uint4 xs = lds_v4(ent_addr + 16u * lq);
-                const uint32_t stage = val_base + d * kStageBytes;
+                // decode role: my 8 words (tile it, word 4h + lgrp at index 2*it + h), their value addresses, the 4 x
                 const unsigned m1 = bit0 << 1, m2 = bit0 << 2, m3 = bit0 << 3;
-                decode_step<0 * kSlotBytes>(w03.x, stage + (off.x & 0xFFFFu), lt_mask, bit0, m1, m2, m3, xs.x, acc[0], acc[1], acc[2], acc[3]);
-                decode_step<0 * kSlotBytes>(w03.y, stage + (off.x >> 16), lt_mask, bit0, m1, m2, m3, xs.x, acc[4], acc[5], acc[6], acc[7]);
-                decode_step<1 * kSlotBytes>(w03.z, stage + (off.y & 0xFFFFu), lt_mask, bit0, m1, m2, m3, xs.y, acc[0], acc[1], acc[2], acc[3]);
-                decode_step<1 * kSlotBytes>(w03.w, stage + (off.y >> 16), lt_mask, bit0, m1, m2, m3, xs.y, acc[4], acc[5], acc[6], acc[7]);
-                decode_step<2 * kSlotBytes>(w47.x, stage + (off.z & 0xFFFFu), lt_mask, bit0, m1, m2, m3, xs.z, acc[0], acc[1], acc[2], acc[3]);
-                decode_step<2 * kSlotBytes>(w47.y, stage + (off.z >> 16), lt_mask, bit0, m1, m2, m3, xs.z, acc[4], acc[5], acc[6], acc[7]);
-                decode_step<3 * kSlotBytes>(w47.z, stage + (off.w & 0xFFFFu), lt_mask, bit0, m1, m2, m3, xs.w, acc[0], acc[1], acc[2], acc[3]);
-                decode_step<3 * kSlotBytes>(w47.w, stage + (off.w >> 16), lt_mask, bit0, m1, m2, m3, xs.w, acc[4], acc[5], acc[6], acc[7]);
+#pragma unroll 1
+                for (int half = 0; half < 2; ++half) {
+                    const uint4 w = lds_v4(bm_dec + d * 128 + 16 * half);
+                    const uint4 a = lds_v4(va_dec + 16 * half);
+                    const uint2 xs = lds_v2(ent_addr + 16u * lq + 8 * half);
+                    decode_step(w.x, a.x, lt_mask, bit0, m1, m2, m3, xs.x, acc[0], acc[1], acc[2], acc[3]);
+                    decode_step(w.y, a.y, lt_mask, bit0, m1, m2, m3, xs.x, acc[4], acc[5], acc[6], acc[7]);
+                    decode_step(w.z, a.z, lt_mask, bit0, m1, m2, m3, xs.y, acc[0], acc[1], acc[2], acc[3]);
+                    decode_step(w.w, a.w, lt_mask, bit0, m1, m2, m3, xs.y, acc[4], acc[5], acc[6], acc[7]);
+                }
                 __syncwarp();                  // everyone is done with ring position d
                 fetch(i + kDepth);
                 d = (d + 1 == kDepth) ? 0 : d + 1;

@@ -18,6 +18,9 @@
 namespace spdp {
 namespace {
 
+#ifndef SPDP_FMA_MODE
+#define SPDP_FMA_MODE 0      // 0: mixed-precision fma.rn.f32.f16, 1: cvt + fp32 fma
+#endif
 #ifndef SPDP_WARPS
 #define SPDP_WARPS 24
 #endif
@@ -63,16 +66,18 @@ struct __align__(128) Smem {
     // [(w & 3) * 8 + it * 2 + (w >> 2)], so the lanes that decode words (w & 3) == g read 8 consecutive words.
     alignas(16) uint32_t bmring[kWarps][kDepth][32];
     alignas(16) uint32_t vaddr[kWarps][32];             // same order: shared address of each word's first value
-    uint32_t colinfo[kChunkCols];                       // ColInfo words of the chunk's GTiles
-    uint32_t tileoff[kChunkGT + 1];                     // TileOffset of the chunk's GTiles
-    alignas(16) uint32_t ent[kChunkCols + kGroup];      // active list: (column in chunk) << 16 | x bits (read 4 at a time)
+    // Active list of the chunk, one record per active column tile (filled once per chunk):
+    alignas(16) uint2 rec[kChunkCols + kGroup];         // .x = start of its values in Values (elements),
+                                                        // .y = (column in chunk) << 6 | 16-byte pieces of values
+    alignas(16) unsigned short xact[kChunkCols + kGroup];   // its activation x_j (fp16 bits)
     uint32_t group_mask[kChunkCols / 32];
     uint32_t group_base[kChunkCols / 32 + 1];
     int is_last;
 };
-static_assert(offsetof(Smem, ent) % 16 == 0 && offsetof(Smem, vaddr) % 16 == 0 && offsetof(Smem, bmring) % 16 == 0,
-              "16-byte shared loads need aligned tables");
+static_assert(offsetof(Smem, rec) % 16 == 0 && offsetof(Smem, xact) % 16 == 0 && offsetof(Smem, vaddr) % 16 == 0 &&
+              offsetof(Smem, bmring) % 16 == 0, "16-byte shared loads need aligned tables");
 static_assert(sizeof(float) * kWarps * kTileM <= size_t(kWarps) * kDepth * kStageBytes, "red must fit in the ring");
+static_assert(sizeof(Smem) <= 227 * 1024, "shared memory of one CTA");
 
 // DP test of Sec. 4.2 step (3): magnitude against the threshold; NOT(|x| <= thr) keeps NaN.
 __device__ __forceinline__ bool column_active(int rule, float thr, const uint32_t* mask, int j, __half xj) {
@@ -128,10 +133,20 @@ __device__ __forceinline__ void decode_step(unsigned W, uint32_t first, unsigned
         " @p1 ld.shared.u16 v1, [a];\n @p1 add.u32 a, a, 2;\n"
         " @p2 ld.shared.u16 v2, [a];\n @p2 add.u32 a, a, 2;\n"
         " @p3 ld.shared.u16 v3, [a];\n"
+#if SPDP_FMA_MODE == 0
         " @p0 fma.rn.f32.f16 %0, v0, xl, %0;\n"
         " @p1 fma.rn.f32.f16 %1, v1, xl, %1;\n"
         " @p2 fma.rn.f32.f16 %2, v2, xl, %2;\n"
         " @p3 fma.rn.f32.f16 %3, v3, xl, %3;\n"
+#else
+        " .reg .f32 f0, f1, f2, f3, fx;\n"
+        " cvt.f32.f16 fx, xl;\n"
+        " @p0 cvt.f32.f16 f0, v0;\n @p1 cvt.f32.f16 f1, v1;\n @p2 cvt.f32.f16 f2, v2;\n @p3 cvt.f32.f16 f3, v3;\n"
+        " @p0 fma.rn.f32 %0, f0, fx, %0;\n"
+        " @p1 fma.rn.f32 %1, f1, fx, %1;\n"
+        " @p2 fma.rn.f32 %2, f2, fx, %2;\n"
+        " @p3 fma.rn.f32 %3, f3, fx, %3;\n"
+#endif
         "}"
         : "+f"(a0), "+f"(a1), "+f"(a2), "+f"(a3)
         : "r"(W), "r"(first), "r"(below), "r"(m0), "r"(m1), "r"(m2), "r"(m3), "r"(x32));
@@ -168,8 +183,8 @@ __device__ __forceinline__ void sts_u32(uint32_t addr, unsigned v) {
 //   (3) segment end: cross-warp row reduction, split-K combine, store.
 __global__ void __launch_bounds__(kThreads, 1)
 spmspv_kernel(const Params p) {
-    extern __shared__ unsigned char smem_raw[];
-    Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    Smem& sm = *reinterpret_cast<Smem*>(smem_raw);
 
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
     const int64_t g_begin = p.cta_begin[blockIdx.x], g_end = p.cta_begin[blockIdx.x + 1];
@@ -189,9 +204,10 @@ spmspv_kernel(const Params p) {
     const uint32_t va_own = smem_u32(&sm.vaddr[warp][tpos]);
     const uint32_t va_dec = smem_u32(&sm.vaddr[warp][lgrp * 8]);
     const uint32_t slot_own = smem_u32(&sm.ring[warp][0][lgrp * kSlotBytes]);      // scan role: my tile's slot
-    const uint32_t ent_addr = smem_u32(&sm.ent[0]);
+    const uint32_t rec_addr = smem_u32(&sm.rec[0]);
+    const uint32_t x_addr = smem_u32(&sm.xact[0]);
     const unsigned char* bm8 = reinterpret_cast<const unsigned char*>(p.bitmap);
-    const unsigned char* val8 = reinterpret_cast<const unsigned char*>(p.values);
+    const unsigned char* val_src = reinterpret_cast<const unsigned char*>(p.values) + 16 * lane7;   // fetch role
 
     for (int64_t g0 = g_begin; g0 < g_end;) {
         const int r = static_cast<int>(g0 / p.C);
@@ -212,9 +228,7 @@ spmspv_kernel(const Params p) {
             const int ngroups32 = (ncols + 31) >> 5;
             const int64_t gt0 = static_cast<int64_t>(r) * p.C + cg;
 
-            // ---- (1) metadata of the chunk and its active-column list ----
-            for (int i = t; i < ngt * kTileK; i += kThreads) sm.colinfo[i] = __ldg(p.colinfo + gt0 * kTileK + i);
-            for (int i = t; i < ngt; i += kThreads) sm.tileoff[i] = __ldg(p.tileoffset + gt0 + i);
+            // ---- (1) active-column list of the chunk (ballots + prefix sums) and its records ----
             for (int q = warp; q < ngroups32; q += kWarps) {
                 const int j = j0 + q * 32 + lane;
                 bool a = false;
@@ -244,8 +258,12 @@ spmspv_kernel(const Params p) {
                 const unsigned m = sm.group_mask[q];
                 if ((m >> lane) & 1u) {
                     const int jj = q * 32 + lane;
-                    const unsigned xb = __half_as_ushort(p.x[j0 + jj]);
-                    sm.ent[sm.group_base[q] + __popc(m & ((1u << lane) - 1u))] = (static_cast<unsigned>(jj) << 16) | xb;
+                    const int item = static_cast<int>(sm.group_base[q] + __popc(m & ((1u << lane) - 1u)));
+                    const uint32_t ci = __ldg(p.colinfo + gt0 * kTileK + jj);               // ColInfo: offset << 16 | nnz
+                    const uint32_t to = __ldg(p.tileoffset + gt0 + (jj >> 4));
+                    sm.rec[item] = make_uint2(to + (ci >> 16),
+                                              (static_cast<unsigned>(jj) << 6) | (((ci & 0xFFFFu) + 7u) >> 3));
+                    sm.xact[item] = __half_as_ushort(p.x[j0 + jj]);
                 }
             }
             __syncthreads();
@@ -262,17 +280,15 @@ spmspv_kernel(const Params p) {
                     const int item = lq * kGroup + lgrp;
                     const uint32_t bdst = bm_own + d * 128;
                     if (item < nact) {
-                        const unsigned jj = sm.ent[item] >> 16;
-                        const uint32_t ci = sm.colinfo[jj];
-                        const int rem = static_cast<int>(((ci & 0xFFFFu) + 7u) >> 3) - lane7;   // my 16-byte pieces left
-                        const unsigned char* src = val8 + 2 * (static_cast<uint64_t>(sm.tileoff[jj >> 4]) + (ci >> 16))
-                                                   + 16 * lane7;
+                        const uint2 rc = lds_v2(rec_addr + 8u * item);
+                        const int rem = static_cast<int>(rc.y & 63u) - lane7;                  // my 16-byte pieces left
+                        const unsigned char* src = val_src + 2 * static_cast<uint64_t>(rc.x);
                         const uint32_t dst = val_dst + d * kStageBytes;
                         cp_async16<0>(dst, src, rem);
                         cp_async16<128>(dst, src, rem);
                         cp_async16<256>(dst, src, rem);
                         cp_async16<384>(dst, src, rem);
-                        cp_async4(bdst, bm_chunk + static_cast<size_t>(jj) * 32);
+                        cp_async4(bdst, bm_chunk + static_cast<size_t>(rc.y >> 6) * 32);
                     } else {
                         sts_u32(bdst, 0u);
                     }
@@ -304,11 +320,11 @@ spmspv_kernel(const Params p) {
                 for (int half = 0; half < 2; ++half) {
                     const uint4 w = lds_v4(bm_dec + d * 128 + 16 * half);
                     const uint4 a = lds_v4(va_dec + 16 * half);
-                    const uint2 xs = lds_v2(ent_addr + 16u * lq + 8 * half);
-                    decode_step(w.x, a.x, lt_mask, bit0, m1, m2, m3, xs.x, acc[0], acc[1], acc[2], acc[3]);
-                    decode_step(w.y, a.y, lt_mask, bit0, m1, m2, m3, xs.x, acc[4], acc[5], acc[6], acc[7]);
-                    decode_step(w.z, a.z, lt_mask, bit0, m1, m2, m3, xs.y, acc[0], acc[1], acc[2], acc[3]);
-                    decode_step(w.w, a.w, lt_mask, bit0, m1, m2, m3, xs.y, acc[4], acc[5], acc[6], acc[7]);
+                    const unsigned xs = lds_u32(x_addr + 8u * lq + 4 * half);        // two activations
+                    decode_step(w.x, a.x, lt_mask, bit0, m1, m2, m3, xs, acc[0], acc[1], acc[2], acc[3]);
+                    decode_step(w.y, a.y, lt_mask, bit0, m1, m2, m3, xs, acc[4], acc[5], acc[6], acc[7]);
+                    decode_step(w.z, a.z, lt_mask, bit0, m1, m2, m3, xs >> 16, acc[0], acc[1], acc[2], acc[3]);
+                    decode_step(w.w, a.w, lt_mask, bit0, m1, m2, m3, xs >> 16, acc[4], acc[5], acc[6], acc[7]);
                 }
                 __syncwarp();                  // everyone is done with ring position d
                 fetch(i + kDepth);
@@ -367,7 +383,7 @@ spmspv_kernel(const Params p) {
 // Launch helper shared by the entry points: opts in to the large dynamic shared memory once per
 // device, then launches P CTAs.
 spdp_status launch_kernel(const Params& p, int num_ctas, cudaStream_t s) {
-    constexpr size_t kSmemBytes = sizeof(Smem) + 128;
+    constexpr size_t kSmemBytes = sizeof(Smem);
     static bool configured[64] = {};
     int dev = 0;
     SPDP_CUDA_TRY(cudaGetDevice(&dev));

@@ -136,8 +136,8 @@ SPDP_API spdp_status spdp_spmspv_host(spdp_handle h, const void* x_host, spdp_dp
  *
  * What spdp_spmspv keeps in handle-owned allocations (CTA ranges, per-row-tile tables, arrival
  * counters, split-K partial sums) lives in ONE fixed device array inside the library, about
- * 0.6 MB, present on every GPU that loads the library until the process exits.  Limits: at most
- * 4096 row tiles (M <= 1,048,576); larger shapes return SPDP_ERR_UNSUPPORTED_SHAPE.  At most 256
+ * 1.1 MB, present on every GPU that loads the library until the process exits.  Limits: at most
+ * 4096 row tiles (M <= 1,048,576); larger shapes return SPDP_ERR_UNSUPPORTED_SHAPE.  At most 512
  * CTAs are launched.  The call enqueues a small set-up kernel (which also clears the counters the
  * previous call left behind) and the spMspV kernel on `stream`; it calls no cudaMalloc, cudaFree or
  * allocating library routine.

@@ -64,7 +64,7 @@ spdp_status new_handle(int64_t M, int64_t K, int pad_elems, spdp_matrix** out) {
 // CTAs feed it.  (Re)allocates the tables, the workspace and the counters.
 spdp_status build_partition(spdp_matrix* h, int num_ctas) {
     const int64_t NGT = h->NGT, C = h->C, R = h->R;
-    int P = num_ctas > 0 ? num_ctas : h->sm_count;
+    int P = num_ctas > 0 ? num_ctas : h->sm_count * default_ctas_per_sm();
     if (P > NGT) P = static_cast<int>(NGT);
     if (P < 1) P = 1;
     std::vector<uint32_t> begin(P + 1);

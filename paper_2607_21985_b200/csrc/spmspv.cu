@@ -24,6 +24,12 @@ namespace {
 #ifndef SPDP_WARPS
 #define SPDP_WARPS 24
 #endif
+#ifndef SPDP_CTAS_PER_SM
+#define SPDP_CTAS_PER_SM 1
+#endif
+#ifndef SPDP_CHUNK_COLS
+#define SPDP_CHUNK_COLS 8192
+#endif
 #ifndef SPDP_DEPTH
 #define SPDP_DEPTH 2
 #endif
@@ -34,7 +40,8 @@ constexpr int kSlotBytes = 2 * kTileM + 32;  // a column tile's values (at most 
                                              // four tiles of a group start 8 banks apart
 constexpr int kStageBytes = kGroup * kSlotBytes;
 constexpr int kThreads = kWarps * 32;
-constexpr int kChunkCols = 8192;           // columns handled between two pipeline drains
+constexpr int kChunkCols = SPDP_CHUNK_COLS; // columns handled between two pipeline drains
+constexpr int kCtasPerSm = SPDP_CTAS_PER_SM;
 constexpr int kChunkGT = kChunkCols / kTileK;
 
 struct Params {
@@ -77,7 +84,7 @@ struct __align__(128) Smem {
 static_assert(offsetof(Smem, rec) % 16 == 0 && offsetof(Smem, xact) % 16 == 0 && offsetof(Smem, vaddr) % 16 == 0 &&
               offsetof(Smem, bmring) % 16 == 0, "16-byte shared loads need aligned tables");
 static_assert(sizeof(float) * kWarps * kTileM <= size_t(kWarps) * kDepth * kStageBytes, "red must fit in the ring");
-static_assert(sizeof(Smem) <= 227 * 1024, "shared memory of one CTA");
+static_assert(sizeof(Smem) <= (227 * 1024) / kCtasPerSm - 1024 * (kCtasPerSm - 1), "shared memory of one CTA");
 
 // DP test of Sec. 4.2 step (3): magnitude against the threshold; NOT(|x| <= thr) keeps NaN.
 __device__ __forceinline__ bool column_active(int rule, float thr, const uint32_t* mask, int j, __half xj) {
@@ -181,7 +188,7 @@ __device__ __forceinline__ void sts_u32(uint32_t addr, unsigned v) {
 //       consecutive rows of a half column tile, rank = set bits before them, values read from
 //       shared memory, fp32 accumulation in registers;
 //   (3) segment end: cross-warp row reduction, split-K combine, store.
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, kCtasPerSm)
 spmspv_kernel(const Params p) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     Smem& sm = *reinterpret_cast<Smem*>(smem_raw);
@@ -415,7 +422,7 @@ __global__ void active_columns_kernel(const __half* __restrict__ x, int K, int r
 // Everything spdp_spmspv keeps in handle-owned allocations (the CTA ranges, the per-row-tile
 // tables, the arrival counters, the split-K partial sums) lives here instead, so the entry point
 // below never allocates.  One copy per device that loads the library, held until exit.
-constexpr int kNoAllocMaxCtas = 256;
+constexpr int kNoAllocMaxCtas = 512;
 constexpr int kNoAllocMaxRowTiles = 4096;          // M <= 1,048,576
 
 struct NoAllocScratch {
@@ -447,6 +454,8 @@ __global__ void noalloc_setup_kernel(NoAllocScratch* sc, int64_t NGT, int64_t C,
 }
 
 }  // namespace
+
+int default_ctas_per_sm() { return kCtasPerSm; }
 
 spdp_status launch_spmspv(const spdp_matrix* h, const __half* x, int rule, float thr,
                           const uint32_t* mask, void* y, int ydt, cudaStream_t s) {
@@ -501,7 +510,7 @@ spdp_status launch_spmspv_noalloc(const uint32_t* tileoffset, const uint32_t* co
         sc = scratch_of[dev];
         sms = sm_count_of[dev];
     }
-    int P = sms < kNoAllocMaxCtas ? sms : kNoAllocMaxCtas;
+    int P = sms * kCtasPerSm < kNoAllocMaxCtas ? sms * kCtasPerSm : kNoAllocMaxCtas;
     if (P > NGT) P = static_cast<int>(NGT);
     noalloc_setup_kernel<<<1, 256, 0, s>>>(sc, NGT, C, static_cast<int>(R), P);
     SPDP_CUDA_TRY(cudaGetLastError());

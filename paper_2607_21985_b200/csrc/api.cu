@@ -215,7 +215,7 @@ spdp_status spdp_spmspv_noalloc(const void* tileoffset_dev, const void* colinfo_
     if (!rule_ok(rule) || (ydt != SPDP_Y_F16 && ydt != SPDP_Y_F32)) return SPDP_ERR_INVALID_ARG;
     if (rule == SPDP_DP_MASK && mask_dev == nullptr) return SPDP_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(values_dev) & 15u) || (reinterpret_cast<uintptr_t>(bitmap_dev) & 7u) ||
-        (reinterpret_cast<uintptr_t>(tileoffset_dev) & 3u) || (reinterpret_cast<uintptr_t>(colinfo_dev) & 3u) ||
+        (reinterpret_cast<uintptr_t>(tileoffset_dev) & 3u) || (reinterpret_cast<uintptr_t>(colinfo_dev) & 15u) ||
         (reinterpret_cast<uintptr_t>(x_dev) & 1u) || (reinterpret_cast<uintptr_t>(mask_dev) & 3u) ||
         (reinterpret_cast<uintptr_t>(y_dev) & (ydt == SPDP_Y_F32 ? 3u : 1u)))
         return SPDP_ERR_INVALID_ARG;

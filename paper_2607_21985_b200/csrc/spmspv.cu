@@ -42,6 +42,7 @@ constexpr int kStageBytes = kGroup * kSlotBytes;
 constexpr int kThreads = kWarps * 32;
 constexpr int kChunkCols = SPDP_CHUNK_COLS; // columns handled between two pipeline drains
 constexpr int kCtasPerSm = SPDP_CTAS_PER_SM;
+constexpr int kListPasses = (kChunkCols / 32 + kWarps - 1) / kWarps;   // 32-column groups a warp scans per chunk
 constexpr int kChunkGT = kChunkCols / kTileK;
 
 struct Params {
@@ -68,6 +69,11 @@ struct __align__(128) Smem {
     union {
         unsigned char ring[kWarps][kDepth][kStageBytes];    // values of the column tiles in flight, per warp
         float red[kWarps][kTileM];                          // cross-warp row reduction (after the pipelines drained)
+        struct {                                            // list phase: the chunk's ColInfo / TileOffset words,
+            float keep_clear_of_red[kWarps][kTileM];        // placed behind red[], which may still be read
+            alignas(16) uint32_t colinfo[kChunkCols];
+            uint32_t tileoff[kChunkGT];
+        } stage;
     };
     // Bitmap words of a group in decode order: word w of the group's it-th tile sits at
     // [(w & 3) * 8 + it * 2 + (w >> 2)], so the lanes that decode words (w & 3) == g read 8 consecutive words.
@@ -84,6 +90,8 @@ struct __align__(128) Smem {
 static_assert(offsetof(Smem, rec) % 16 == 0 && offsetof(Smem, xact) % 16 == 0 && offsetof(Smem, vaddr) % 16 == 0 &&
               offsetof(Smem, bmring) % 16 == 0, "16-byte shared loads need aligned tables");
 static_assert(sizeof(float) * kWarps * kTileM <= size_t(kWarps) * kDepth * kStageBytes, "red must fit in the ring");
+static_assert(sizeof(uint32_t) * (kChunkCols + kChunkGT) + sizeof(float) * kWarps * kTileM <= size_t(kWarps) * kDepth * kStageBytes,
+              "staging must fit in the ring behind red");
 static_assert(sizeof(Smem) <= (227 * 1024) / kCtasPerSm - 1024 * (kCtasPerSm - 1), "shared memory of one CTA");
 
 // DP test of Sec. 4.2 step (3): magnitude against the threshold; NOT(|x| <= thr) keeps NaN.
@@ -236,13 +244,43 @@ spmspv_kernel(const Params p) {
             const int64_t gt0 = static_cast<int64_t>(r) * p.C + cg;
 
             // ---- (1) active-column list of the chunk (ballots + prefix sums) and its records ----
-            for (int q = warp; q < ngroups32; q += kWarps) {
+            // One memory round trip: the chunk's ColInfo and TileOffset words stream into the idle
+            // ring with asynchronous copies while x is read and tested.  ColInfo of skipped columns
+            // is read too (4 bytes per column tile); their bitmaps and values never are.
+            {
+                const uint32_t ci_stage = smem_u32(&sm.stage.colinfo[0]);
+                const uint32_t to_stage = smem_u32(&sm.stage.tileoff[0]);
+                const uint4* ci_src = reinterpret_cast<const uint4*>(p.colinfo + gt0 * kTileK);
+                for (int i = t; i < ngt * (kTileK / 4); i += kThreads) cp_async16<0>(ci_stage + 16 * i, ci_src + i, 1);
+                for (int i = t; i < ngt; i += kThreads) cp_async4(to_stage + 4 * i, p.tileoffset + gt0 + i);
+                cp_async_commit();
+            }
+            unsigned xb[kListPasses], act[kListPasses];
+#pragma unroll
+            for (int u = 0; u < kListPasses; ++u) {
+                const int j = j0 + (warp + u * kWarps) * 32 + lane;
+                xb[u] = 0u;
+                act[u] = 0u;
+                if (j < j_hi) {
+                    xb[u] = __half_as_ushort(p.x[j]);
+                    if (p.rule == SPDP_DP_MASK) act[u] = __ldg(p.mask + (j >> 5));
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < kListPasses; ++u) {
+                const int q = warp + u * kWarps;
                 const int j = j0 + q * 32 + lane;
                 bool a = false;
-                if (j < j_hi) a = column_active(p.rule, p.thr, p.mask, j, p.x[j]);
-                const unsigned m = __ballot_sync(0xFFFFFFFFu, a);
-                if (lane == 0) sm.group_mask[q] = m;
+                if (j < j_hi) {
+                    if (p.rule == SPDP_DP_NONE) a = true;
+                    else if (p.rule == SPDP_DP_ABS_GT)
+                        a = !(fabsf(__half2float(__ushort_as_half(static_cast<unsigned short>(xb[u])))) <= p.thr);
+                    else a = (act[u] >> (j & 31)) & 1u;
+                }
+                act[u] = __ballot_sync(0xFFFFFFFFu, a);
+                if (lane == 0 && q < ngroups32) sm.group_mask[q] = act[u];
             }
+            cp_async_wait<0>();
             __syncthreads();
             if (warp == 0) {
                 unsigned run = 0;
@@ -261,19 +299,19 @@ spmspv_kernel(const Params p) {
                 if (lane == 0) sm.group_base[ngroups32] = run;
             }
             __syncthreads();
-            for (int q = warp; q < ngroups32; q += kWarps) {
-                const unsigned m = sm.group_mask[q];
-                if ((m >> lane) & 1u) {
+#pragma unroll
+            for (int u = 0; u < kListPasses; ++u) {
+                const int q = warp + u * kWarps;
+                if ((act[u] >> lane) & 1u) {
                     const int jj = q * 32 + lane;
-                    const int item = static_cast<int>(sm.group_base[q] + __popc(m & ((1u << lane) - 1u)));
-                    const uint32_t ci = __ldg(p.colinfo + gt0 * kTileK + jj);               // ColInfo: offset << 16 | nnz
-                    const uint32_t to = __ldg(p.tileoffset + gt0 + (jj >> 4));
-                    sm.rec[item] = make_uint2(to + (ci >> 16),
+                    const int item = static_cast<int>(sm.group_base[q] + __popc(act[u] & ((1u << lane) - 1u)));
+                    const uint32_t ci = sm.stage.colinfo[jj];                           // ColInfo: offset << 16 | nnz
+                    sm.rec[item] = make_uint2(sm.stage.tileoff[jj >> 4] + (ci >> 16),
                                               (static_cast<unsigned>(jj) << 6) | (((ci & 0xFFFFu) + 7u) >> 3));
-                    sm.xact[item] = __half_as_ushort(p.x[j0 + jj]);
+                    sm.xact[item] = static_cast<unsigned short>(xb[u]);
                 }
             }
-            __syncthreads();
+            __syncthreads();       // the records are complete; the staging area becomes the ring again
             const int nact = static_cast<int>(sm.group_base[ngroups32]);
             const int ngroups = (nact + kGroup - 1) / kGroup;
 
@@ -348,42 +386,45 @@ spmspv_kernel(const Params p) {
             sm.red[warp][128 + 4 * lane + k] = acc[4 + k];
         }
         __syncthreads();
-        float part = 0.f;
-        const int64_t row = static_cast<int64_t>(r) * kTileM + t;
+        // The first 256 threads (one per row) finish the segment; the other warps go straight on to
+        // the next segment's list phase, whose global loads overlap the combine.  The ring is not
+        // written again before the next __syncthreads, which these 256 threads join afterwards.
         if (t < kTileM) {
+            float part = 0.f;
+            const int64_t row = static_cast<int64_t>(r) * kTileM + t;
 #pragma unroll
             for (int w = 0; w < kWarps; ++w) part += sm.red[w][t];
-        }
-        // ---- split-K combine ----
-        const int nseg = p.row_nseg[r];
-        if (nseg == 1) {
-            if (t < kTileM && row < p.M) store_y(p.y, p.ydt, row, part);
-        } else {
-            float* mine = p.workspace + (static_cast<int64_t>(blockIdx.x) * 2 + (r != r_first)) * kTileM;
-            if (t < kTileM) __stcg(mine + t, part);
-            __threadfence();
-            __syncthreads();
-            if (t == 0) {
-                const unsigned old = atomicAdd(p.row_counter + r, 1u);
-                sm.is_last = (old == static_cast<unsigned>(nseg - 1));
-            }
-            __syncthreads();
-            if (sm.is_last) {
+            // ---- split-K combine ----
+            const int nseg = p.row_nseg[r];
+            if (nseg == 1) {
+                if (row < p.M) store_y(p.y, p.ydt, row, part);
+            } else {
+                float* mine = p.workspace + (static_cast<int64_t>(blockIdx.x) * 2 + (r != r_first)) * kTileM;
+                __stcg(mine + t, part);
                 __threadfence();
-                if (t < kTileM && row < p.M) {
-                    const int q0 = p.row_first_cta[r];
-                    float sum = 0.f;
-                    for (int s = 0; s < nseg; ++s) {
-                        const int q = q0 + s;
-                        const int slot = (r != static_cast<int>(p.cta_begin[q] / p.C));
-                        sum += __ldcg(p.workspace + (static_cast<int64_t>(q) * 2 + slot) * kTileM + t);
-                    }
-                    store_y(p.y, p.ydt, row, sum);
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+                if (t == 0) {
+                    const unsigned old = atomicAdd(p.row_counter + r, 1u);
+                    sm.is_last = (old == static_cast<unsigned>(nseg - 1));
                 }
-                if (t == 0) p.row_counter[r] = 0;       // ready for the next call on this handle
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+                if (sm.is_last) {
+                    __threadfence();
+                    if (row < p.M) {
+                        const int q0 = p.row_first_cta[r];
+                        float sum = 0.f;
+                        for (int s = 0; s < nseg; ++s) {
+                            const int q = q0 + s;
+                            const int slot = (r != static_cast<int>(p.cta_begin[q] / p.C));
+                            sum += __ldcg(p.workspace + (static_cast<int64_t>(q) * 2 + slot) * kTileM + t);
+                        }
+                        store_y(p.y, p.ydt, row, sum);
+                    }
+                    if (t == 0) p.row_counter[r] = 0;       // ready for the next call on this handle
+                }
+                asm volatile("bar.sync 1, 256;" ::: "memory");   // is_last is rewritten by the next segment
             }
         }
-        __syncthreads();           // red[] (the ring) and is_last are reused by the next segment
     }
 }
 

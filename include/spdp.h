@@ -81,7 +81,9 @@ typedef struct {
  *   W_dev     fp16 [M][ldw] row-major, device; an element is "pruned" iff its value is +-0
  *             (bits & 0x7FFF == 0); every other bit pattern, NaN/Inf/subnormals included, is
  *             stored verbatim.
- *   M, K      >= 1; sides that are not multiples of 256 / 16 are zero-extended logically.
+ *   M, K      >= 1; sides that are not multiples of 256 / 16 are zero-extended logically.  The matrix
+ *             may hold at most 2^26 column tiles (ceil(M/256) * ceil(K/16) * 16), else
+ *             SPDP_ERR_UNSUPPORTED_SHAPE.
  *   ldw       leading dimension in elements, >= K.
  *   tile_m, tile_k  must be 256 and 16 (the format's constants), else SPDP_ERR_UNSUPPORTED_SHAPE.
  *   out       receives the handle.  The call allocates device memory, runs on `stream` and

@@ -52,7 +52,8 @@ spdp_status new_handle(int64_t M, int64_t K, int pad_elems, spdp_matrix** out) {
     h->C = (K + kTileK - 1) / kTileK;
     h->NGT = h->R * h->C;
     h->pad_elems = pad_elems;
-    if (h->NGT >= (int64_t(1) << 31) / kTileK) { delete h; return SPDP_ERR_UNSUPPORTED_SHAPE; }
+    // the kernel packs a column-tile index and a 6-bit count into 32 bits
+    if (h->NGT * kTileK >= (int64_t(1) << 26)) { delete h; return SPDP_ERR_UNSUPPORTED_SHAPE; }
     cudaError_t e = cudaGetDevice(&h->device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->sm_count, cudaDevAttrMultiProcessorCount, h->device);
     if (e != cudaSuccess) { note_cuda_error(e, "device query"); delete h; return SPDP_ERR_CUDA; }

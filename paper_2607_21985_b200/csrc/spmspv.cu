@@ -42,7 +42,7 @@ constexpr int kStageBytes = kGroup * kSlotBytes;
 constexpr int kThreads = kWarps * 32;
 constexpr int kChunkCols = SPDP_CHUNK_COLS; // columns handled between two pipeline drains
 constexpr int kCtasPerSm = SPDP_CTAS_PER_SM;
-constexpr int kListPasses = (kChunkCols / 32 + kWarps - 1) / kWarps;   // 32-column groups a warp scans per chunk
+constexpr uint32_t kNullRec = 0xFFFFFFFFu;
 constexpr int kChunkGT = kChunkCols / kTileK;
 
 struct Params {
@@ -72,6 +72,7 @@ struct __align__(128) Smem {
         struct {                                            // list phase: the chunk's ColInfo / TileOffset words,
             float keep_clear_of_red[kWarps][kTileM];        // placed behind red[], which may still be read
             alignas(16) uint32_t colinfo[kChunkCols];
+            alignas(16) unsigned short x[kChunkCols];       // and the activations of the listed columns
             uint32_t tileoff[kChunkGT];
         } stage;
     };
@@ -81,18 +82,22 @@ struct __align__(128) Smem {
     alignas(16) uint32_t vaddr[kWarps][32];             // same order: shared address of each word's first value
     // Active list of the chunk, one record per active column tile (filled once per chunk):
     alignas(16) uint2 rec[kChunkCols + kGroup];         // .x = start of its values in Values (elements),
-                                                        // .y = (column in chunk) << 6 | 16-byte pieces of values
+                                                        // .y = (column slot in Bitmap/ColInfo) << 6 | 16-byte pieces
+                                                        //      of values; kNullRec pads a piece to whole groups
     alignas(16) unsigned short xact[kChunkCols + kGroup];   // its activation x_j (fp16 bits)
+    float red_first[kWarps][kTileM];                    // row reduction of a batch's first piece (flushed mid-stream)
     uint32_t group_mask[kChunkCols / 32];
     uint32_t group_base[kChunkCols / 32 + 1];
-    int is_last;
+    int is_last[2];
 };
 static_assert(offsetof(Smem, rec) % 16 == 0 && offsetof(Smem, xact) % 16 == 0 && offsetof(Smem, vaddr) % 16 == 0 &&
               offsetof(Smem, bmring) % 16 == 0, "16-byte shared loads need aligned tables");
 static_assert(sizeof(float) * kWarps * kTileM <= size_t(kWarps) * kDepth * kStageBytes, "red must fit in the ring");
-static_assert(sizeof(uint32_t) * (kChunkCols + kChunkGT) + sizeof(float) * kWarps * kTileM <= size_t(kWarps) * kDepth * kStageBytes,
+static_assert(sizeof(uint32_t) * (kChunkCols + kChunkGT) + 2 * kChunkCols + sizeof(float) * kWarps * kTileM <=
+                  size_t(kWarps) * kDepth * kStageBytes,
               "staging must fit in the ring behind red");
 static_assert(sizeof(Smem) <= (227 * 1024) / kCtasPerSm - 1024 * (kCtasPerSm - 1), "shared memory of one CTA");
+static_assert(kWarps >= 16, "two groups of 256 threads finish two row tiles side by side");
 
 // DP test of Sec. 4.2 step (3): magnitude against the threshold; NOT(|x| <= thr) keeps NaN.
 __device__ __forceinline__ bool column_active(int rule, float thr, const uint32_t* mask, int j, __half xj) {
@@ -114,6 +119,10 @@ template <int kOff>
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int rem) {
     asm volatile("{\n .reg .pred p;\n setp.gt.s32 p, %2, %3;\n @p cp.async.cg.shared.global [%0+%4], [%1+%4], 16;\n}"
                  ::"r"(dst), "l"(src), "r"(rem), "n"(kOff / 16), "n"(kOff) : "memory");
+}
+// 16-byte copy that reads only the first `bytes` (0..16) source bytes and zero-fills the rest.
+__device__ __forceinline__ void cp_async16_partial(uint32_t dst, const void* src, int bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ void cp_async4(uint32_t dst, const void* src) {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
@@ -185,17 +194,62 @@ __device__ __forceinline__ void sts_u32(uint32_t addr, unsigned v) {
     asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
 
+// Adds the kWarps per-warp partial sums of one row tile in warp order and finishes the row tile
+// (256 threads, tt = row inside the tile, `bar` = a named barrier of these 256 threads).  A row tile
+// fed by one segment is stored directly; otherwise the sum goes to this CTA's workspace slot and
+// the CTA that arrives last at the row tile's counter adds all partials in CTA order.
+__device__ __forceinline__ void finish_row_tile(const Params& p, int r, int r_first, const float (*red)[kTileM],
+                                                int tt, int bar, int* is_last) {
+    float part = 0.f;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) part += red[w][tt];
+    const int64_t row = static_cast<int64_t>(r) * kTileM + tt;
+    const int nseg = p.row_nseg[r];
+    if (nseg == 1) {
+        if (row < p.M) store_y(p.y, p.ydt, row, part);
+        return;
+    }
+    __stcg(p.workspace + (static_cast<int64_t>(blockIdx.x) * 2 + (r != r_first)) * kTileM + tt, part);
+    __threadfence();
+    asm volatile("bar.sync %0, 256;" ::"r"(bar) : "memory");
+    if (tt == 0) {
+        const unsigned old = atomicAdd(p.row_counter + r, 1u);
+        *is_last = (old == static_cast<unsigned>(nseg - 1));
+    }
+    asm volatile("bar.sync %0, 256;" ::"r"(bar) : "memory");
+    if (*is_last) {
+        __threadfence();
+        if (row < p.M) {
+            const int q0 = p.row_first_cta[r];
+            float sum = 0.f;
+            for (int s = 0; s < nseg; ++s) {
+                const int q = q0 + s;
+                const int slot = (r != static_cast<int>(p.cta_begin[q] / p.C));
+                sum += __ldcg(p.workspace + (static_cast<int64_t>(q) * 2 + slot) * kTileM + tt);
+            }
+            store_y(p.y, p.ydt, row, sum);
+        }
+        if (tt == 0) p.row_counter[r] = 0;          // ready for the next call on this handle
+    }
+    asm volatile("bar.sync %0, 256;" ::"r"(bar) : "memory");       // is_last may be rewritten by the next batch
+}
+
 // One persistent CTA per GTile range; every warp runs its own fetch -> decode pipeline.
-// Per chunk of the range:
-//   (1) all warps: ColInfo / TileOffset of the chunk to shared memory and the active-column list
-//       from x (ballots + prefix sums) -- Sec. 4.2 steps (1)-(3);
+// The range is cut into pieces (part of one row tile, at most kChunkGT GTiles).  A batch is one
+// piece, or the last piece of a row tile together with the first piece of the next row tile, so
+// that the usual CTA range (the tail of one row tile and the head of the next) is one batch.
+// Per batch:
+//   (1) all warps: the pieces' ColInfo / TileOffset words and the active-column list from x
+//       (ballots + prefix sums), one record per active column tile -- Sec. 4.2 steps (1)-(3);
 //   (2) each warp takes groups of kGroup active column tiles round-robin.  It keeps kDepth
 //       groups in flight: the padded values of a column tile arrive with 16-byte asynchronous
 //       copies (lane = one 16-byte piece of one of the group's tiles), its 8 bitmap words with
 //       4-byte ones; inactive columns are never touched.  Decode (Sec. 4.2.1): lane owns 4
 //       consecutive rows of a half column tile, rank = set bits before them, values read from
-//       shared memory, fp32 accumulation in registers;
-//   (3) segment end: cross-warp row reduction, split-K combine, store.
+//       shared memory, fp32 accumulation in registers.  Where the first piece's groups end the
+//       warp parks its sums in shared memory and starts the second piece from zero;
+//   (3) batch end: cross-warp row reduction, split-K combine and store of every row tile that
+//       the batch completed (two groups of 256 threads work side by side).
 __global__ void __launch_bounds__(kThreads, kCtasPerSm)
 spmspv_kernel(const Params p) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -221,209 +275,257 @@ spmspv_kernel(const Params p) {
     const uint32_t slot_own = smem_u32(&sm.ring[warp][0][lgrp * kSlotBytes]);      // scan role: my tile's slot
     const uint32_t rec_addr = smem_u32(&sm.rec[0]);
     const uint32_t x_addr = smem_u32(&sm.xact[0]);
-    const unsigned char* bm8 = reinterpret_cast<const unsigned char*>(p.bitmap);
+    const unsigned char* bm_src = reinterpret_cast<const unsigned char*>(p.bitmap) + lane7 * 4;     // fetch role
     const unsigned char* val_src = reinterpret_cast<const unsigned char*>(p.values) + 16 * lane7;   // fetch role
 
+    float acc[8];                   // rows 4*lane+k (k<4) and 128+4*lane+(k-4) of the current row tile
+#pragma unroll
+    for (int k = 0; k < 8; ++k) acc[k] = 0.f;
+
     for (int64_t g0 = g_begin; g0 < g_end;) {
-        const int r = static_cast<int>(g0 / p.C);
-        const int c_lo = static_cast<int>(g0 - static_cast<int64_t>(r) * p.C);
-        const int64_t c_end = c_lo + (g_end - g0);
-        const int c_hi = static_cast<int>(c_end < p.C ? c_end : p.C);
-        g0 += c_hi - c_lo;
-
-        float acc[8];                   // rows 4*lane+k (k<4) and 128+4*lane+(k-4) of the row tile
-#pragma unroll
-        for (int k = 0; k < 8; ++k) acc[k] = 0.f;
-
-        const int64_t row_slot0 = static_cast<int64_t>(r) * p.C * kTileK;       // column slot of column 0
-        for (int cg = c_lo; cg < c_hi; cg += kChunkGT) {
-            const int ngt = min(kChunkGT, c_hi - cg);
-            const int j0 = cg * kTileK, j_hi = min((cg + ngt) * kTileK, p.K);
-            const int ncols = j_hi - j0;
-            const int ngroups32 = (ncols + 31) >> 5;
-            const int64_t gt0 = static_cast<int64_t>(r) * p.C + cg;
-
-            // ---- (1) active-column list of the chunk (ballots + prefix sums) and its records ----
-            // One memory round trip: the chunk's ColInfo and TileOffset words stream into the idle
-            // ring with asynchronous copies while x is read and tested.  ColInfo of skipped columns
-            // is read too (4 bytes per column tile); their bitmaps and values never are.
-            {
-                const uint32_t ci_stage = smem_u32(&sm.stage.colinfo[0]);
-                const uint32_t to_stage = smem_u32(&sm.stage.tileoff[0]);
-                const uint4* ci_src = reinterpret_cast<const uint4*>(p.colinfo + gt0 * kTileK);
-                for (int i = t; i < ngt * (kTileK / 4); i += kThreads) cp_async16<0>(ci_stage + 16 * i, ci_src + i, 1);
-                for (int i = t; i < ngt; i += kThreads) cp_async4(to_stage + 4 * i, p.tileoffset + gt0 + i);
-                cp_async_commit();
-            }
-            unsigned xb[kListPasses], act[kListPasses];
-#pragma unroll
-            for (int u = 0; u < kListPasses; ++u) {
-                const int j = j0 + (warp + u * kWarps) * 32 + lane;
-                xb[u] = 0u;
-                act[u] = 0u;
-                if (j < j_hi) {
-                    xb[u] = __half_as_ushort(p.x[j]);
-                    if (p.rule == SPDP_DP_MASK) act[u] = __ldg(p.mask + (j >> 5));
-                }
-            }
-#pragma unroll
-            for (int u = 0; u < kListPasses; ++u) {
-                const int q = warp + u * kWarps;
-                const int j = j0 + q * 32 + lane;
-                bool a = false;
-                if (j < j_hi) {
-                    if (p.rule == SPDP_DP_NONE) a = true;
-                    else if (p.rule == SPDP_DP_ABS_GT)
-                        a = !(fabsf(__half2float(__ushort_as_half(static_cast<unsigned short>(xb[u])))) <= p.thr);
-                    else a = (act[u] >> (j & 31)) & 1u;
-                }
-                act[u] = __ballot_sync(0xFFFFFFFFu, a);
-                if (lane == 0 && q < ngroups32) sm.group_mask[q] = act[u];
-            }
-            cp_async_wait<0>();
-            __syncthreads();
-            if (warp == 0) {
-                unsigned run = 0;
-                for (int q0 = 0; q0 < ngroups32; q0 += 32) {
-                    const int q = q0 + lane;
-                    unsigned c = (q < ngroups32) ? __popc(sm.group_mask[q]) : 0u;
-                    unsigned inc = c;
-#pragma unroll
-                    for (int d = 1; d < 32; d <<= 1) {
-                        unsigned v = __shfl_up_sync(0xFFFFFFFFu, inc, d);
-                        if (lane >= d) inc += v;
-                    }
-                    if (q < ngroups32) sm.group_base[q] = run + inc - c;
-                    run += __shfl_sync(0xFFFFFFFFu, inc, 31);
-                }
-                if (lane == 0) sm.group_base[ngroups32] = run;
-            }
-            __syncthreads();
-#pragma unroll
-            for (int u = 0; u < kListPasses; ++u) {
-                const int q = warp + u * kWarps;
-                if ((act[u] >> lane) & 1u) {
-                    const int jj = q * 32 + lane;
-                    const int item = static_cast<int>(sm.group_base[q] + __popc(act[u] & ((1u << lane) - 1u)));
-                    const uint32_t ci = sm.stage.colinfo[jj];                           // ColInfo: offset << 16 | nnz
-                    sm.rec[item] = make_uint2(sm.stage.tileoff[jj >> 4] + (ci >> 16),
-                                              (static_cast<unsigned>(jj) << 6) | (((ci & 0xFFFFu) + 7u) >> 3));
-                    sm.xact[item] = static_cast<unsigned short>(xb[u]);
-                }
-            }
-            __syncthreads();       // the records are complete; the staging area becomes the ring again
-            const int nact = static_cast<int>(sm.group_base[ngroups32]);
-            const int ngroups = (nact + kGroup - 1) / kGroup;
-
-            // ---- (2) per-warp fetch / decode pipeline over groups warp, warp + kWarps, ... ----
-            const unsigned char* bm_chunk = bm8 + (row_slot0 + j0) * 32 + lane7 * 4;
-            // fetch(i): start the copies of my i-th group into ring position i % kDepth
-            auto fetch = [&](int i) {
-                const int lq = warp + i * kWarps;
-                if (lq < ngroups) {
-                    const int d = i % kDepth;
-                    const int item = lq * kGroup + lgrp;
-                    const uint32_t bdst = bm_own + d * 128;
-                    if (item < nact) {
-                        const uint2 rc = lds_v2(rec_addr + 8u * item);
-                        const int rem = static_cast<int>(rc.y & 63u) - lane7;                  // my 16-byte pieces left
-                        const unsigned char* src = val_src + 2 * static_cast<uint64_t>(rc.x);
-                        const uint32_t dst = val_dst + d * kStageBytes;
-                        cp_async16<0>(dst, src, rem);
-                        cp_async16<128>(dst, src, rem);
-                        cp_async16<256>(dst, src, rem);
-                        cp_async16<384>(dst, src, rem);
-                        cp_async4(bdst, bm_chunk + static_cast<size_t>(rc.y >> 6) * 32);
-                    } else {
-                        sts_u32(bdst, 0u);
-                    }
-                }
-                cp_async_commit();
-            };
-#pragma unroll
-            for (int d = 0; d < kDepth; ++d) fetch(d);
-
-            int d = 0;
-            for (int i = 0, lq = warp; lq < ngroups; ++i, lq += kWarps) {
-                cp_async_wait<kDepth - 1>();
-                __syncwarp();
-                // scan role: shared address of my word's first value
-                {
-                    const unsigned cnt = __popc(lds_u32(bm_own + d * 128));
-                    unsigned inc = cnt;
-#pragma unroll
-                    for (int dd = 1; dd < 8; dd <<= 1) {
-                        unsigned v = __shfl_up_sync(0xFFFFFFFFu, inc, dd, 8);
-                        if (lane7 >= dd) inc += v;
-                    }
-                    sts_u32(va_own, slot_own + d * kStageBytes + 2u * (inc - cnt));
-                }
-                __syncwarp();
-                // decode role: my 8 words (tile it, word 4h + lgrp at index 2*it + h), their value addresses, the 4 x
-                const unsigned m1 = bit0 << 1, m2 = bit0 << 2, m3 = bit0 << 3;
-#pragma unroll 1
-                for (int half = 0; half < 2; ++half) {
-                    const uint4 w = lds_v4(bm_dec + d * 128 + 16 * half);
-                    const uint4 a = lds_v4(va_dec + 16 * half);
-                    const unsigned xs = lds_u32(x_addr + 8u * lq + 4 * half);        // two activations
-                    decode_step(w.x, a.x, lt_mask, bit0, m1, m2, m3, xs, acc[0], acc[1], acc[2], acc[3]);
-                    decode_step(w.y, a.y, lt_mask, bit0, m1, m2, m3, xs, acc[4], acc[5], acc[6], acc[7]);
-                    decode_step(w.z, a.z, lt_mask, bit0, m1, m2, m3, xs >> 16, acc[0], acc[1], acc[2], acc[3]);
-                    decode_step(w.w, a.w, lt_mask, bit0, m1, m2, m3, xs >> 16, acc[4], acc[5], acc[6], acc[7]);
-                }
-                __syncwarp();                  // everyone is done with ring position d
-                fetch(i + kDepth);
-                d = (d + 1 == kDepth) ? 0 : d + 1;
-            }
-            cp_async_wait<0>();
-            __syncthreads();       // the chunk's shared tables are rebuilt next; the ring is idle
+        // ---- the batch: piece A = [gA, gA + ngtA) of row tile rA, optionally piece B of row tile rA + 1 ----
+        const int rA = static_cast<int>(g0 / p.C);
+        const int cA = static_cast<int>(g0 - static_cast<int64_t>(rA) * p.C);
+        int ngtA = p.C - cA;
+        if (ngtA > g_end - g0) ngtA = static_cast<int>(g_end - g0);
+        if (ngtA > kChunkGT) ngtA = kChunkGT;
+        const int64_t gA = g0;
+        g0 += ngtA;
+        const bool doneA = (cA + ngtA == p.C) || (g0 == g_end);     // piece A ends its row tile's share of this CTA
+        const int jA0 = cA * kTileK;
+        const int nA = min((cA + ngtA) * kTileK, p.K) - jA0;         // columns of piece A
+        const int vB0 = (ngtA * kTileK + 31) & ~31;                  // piece B starts at this list position
+        int ngtB = 0, nB = 0;
+        bool doneB = false;
+        if (doneA && g0 < g_end && cA + ngtA == p.C) {
+            ngtB = p.C;
+            if (ngtB > g_end - g0) ngtB = static_cast<int>(g_end - g0);
+            if (ngtB > (kChunkCols - vB0) / kTileK) ngtB = (kChunkCols - vB0) / kTileK;
+            nB = min(ngtB * kTileK, p.K);
+            doneB = (ngtB == p.C) || (g0 + ngtB == g_end);
         }
+        const int64_t gB = g0;
+        g0 += ngtB;
+        const int rB = rA + 1;
+        const int nlist = (ngtB > 0) ? vB0 + nB : nA;               // list positions (A, padding, B)
+        const int ngroups32 = (nlist + 31) >> 5;
+        const int qB = (ngtB > 0) ? (vB0 >> 5) : ngroups32;         // first 32-position group of piece B
 
-        // ---- (3) row reduction across the warps (fixed order); red[] reuses the idle ring ----
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            sm.red[warp][4 * lane + k] = acc[k];
-            sm.red[warp][128 + 4 * lane + k] = acc[4 + k];
+        // ---- (1) active-column list of the batch (ballots + prefix sums) and its records ----
+        // One memory round trip: the pieces' ColInfo and TileOffset words and their slice of x stream
+        // into the idle ring with asynchronous copies.  ColInfo of skipped columns is read too
+        // (4 bytes per column tile); their bitmaps and values never are.
+        {
+            const uint32_t ci_stage = smem_u32(&sm.stage.colinfo[0]);
+            const uint32_t to_stage = smem_u32(&sm.stage.tileoff[0]);
+            const uint32_t x_stage = smem_u32(&sm.stage.x[0]);
+            const uint4* ciA = reinterpret_cast<const uint4*>(p.colinfo + gA * kTileK);
+            const uint4* ciB = reinterpret_cast<const uint4*>(p.colinfo + gB * kTileK);
+            for (int i = t; i < ngtA * (kTileK / 4); i += kThreads) cp_async16<0>(ci_stage + 16 * i, ciA + i, 1);
+            for (int i = t; i < ngtB * (kTileK / 4); i += kThreads) cp_async16<0>(ci_stage + 4 * vB0 + 16 * i, ciB + i, 1);
+            for (int i = t; i < ngtA; i += kThreads) cp_async4(to_stage + 4 * i, p.tileoffset + gA + i);
+            for (int i = t; i < ngtB; i += kThreads) cp_async4(to_stage + (vB0 >> 2) + 4 * i, p.tileoffset + gB + i);
+            if ((reinterpret_cast<uintptr_t>(p.x) & 15u) == 0) {
+                // list position v holds x[jA0 + v] (piece A) or x[v - vB0] (piece B); 8 activations per copy
+                for (int i = t; 8 * i < nA; i += kThreads)
+                    cp_async16_partial(x_stage + 16 * i, p.x + jA0 + 8 * i, 2 * min(8, nA - 8 * i));
+                for (int i = t; 8 * i < nB; i += kThreads)
+                    cp_async16_partial(x_stage + 2 * vB0 + 16 * i, p.x + 8 * i, 2 * min(8, nB - 8 * i));
+            } else {
+                for (int v = t; v < nA; v += kThreads) sm.stage.x[v] = __half_as_ushort(p.x[jA0 + v]);
+                for (int v = t; v < nB; v += kThreads) sm.stage.x[vB0 + v] = __half_as_ushort(p.x[v]);
+            }
+            cp_async_commit();
+        }
+        cp_async_wait<0>();
+        __syncthreads();
+#pragma unroll 4
+        for (int q = warp; q < ngroups32; q += kWarps) {
+            const int v = q * 32 + lane;                             // list position
+            const int j = (v < vB0) ? jA0 + v : v - vB0;             // its column
+            bool a = (v < vB0) ? (v < nA) : (v < nlist);
+            if (a) {
+                if (p.rule == SPDP_DP_ABS_GT)
+                    a = !(fabsf(__half2float(__ushort_as_half(sm.stage.x[v]))) <= p.thr);
+                else if (p.rule == SPDP_DP_MASK)
+                    a = (__ldg(p.mask + (j >> 5)) >> (j & 31)) & 1u;
+            }
+            const unsigned m = __ballot_sync(0xFFFFFFFFu, a);
+            if (lane == 0) sm.group_mask[q] = m;
         }
         __syncthreads();
-        // The first 256 threads (one per row) finish the segment; the other warps go straight on to
-        // the next segment's list phase, whose global loads overlap the combine.  The ring is not
-        // written again before the next __syncthreads, which these 256 threads join afterwards.
-        if (t < kTileM) {
-            float part = 0.f;
-            const int64_t row = static_cast<int64_t>(r) * kTileM + t;
+        if (warp == 0) {
+            // Exclusive prefix sums of the group counts: lane l owns groups [l*per, (l+1)*per).  Piece B
+            // starts on a whole group of kGroup records: the padding is counted in front of its first group.
+            constexpr int kMaxPer = (kChunkCols / 32 + 31) / 32;
+            const int per = (ngroups32 + 31) >> 5;
+            unsigned cnt[kMaxPer];
+            unsigned mine = 0, beforeB = 0;
 #pragma unroll
-            for (int w = 0; w < kWarps; ++w) part += sm.red[w][t];
-            // ---- split-K combine ----
-            const int nseg = p.row_nseg[r];
-            if (nseg == 1) {
-                if (row < p.M) store_y(p.y, p.ydt, row, part);
-            } else {
-                float* mine = p.workspace + (static_cast<int64_t>(blockIdx.x) * 2 + (r != r_first)) * kTileM;
-                __stcg(mine + t, part);
-                __threadfence();
-                asm volatile("bar.sync 1, 256;" ::: "memory");
-                if (t == 0) {
-                    const unsigned old = atomicAdd(p.row_counter + r, 1u);
-                    sm.is_last = (old == static_cast<unsigned>(nseg - 1));
-                }
-                asm volatile("bar.sync 1, 256;" ::: "memory");
-                if (sm.is_last) {
-                    __threadfence();
-                    if (row < p.M) {
-                        const int q0 = p.row_first_cta[r];
-                        float sum = 0.f;
-                        for (int s = 0; s < nseg; ++s) {
-                            const int q = q0 + s;
-                            const int slot = (r != static_cast<int>(p.cta_begin[q] / p.C));
-                            sum += __ldcg(p.workspace + (static_cast<int64_t>(q) * 2 + slot) * kTileM + t);
-                        }
-                        store_y(p.y, p.ydt, row, sum);
-                    }
-                    if (t == 0) p.row_counter[r] = 0;       // ready for the next call on this handle
-                }
-                asm volatile("bar.sync 1, 256;" ::: "memory");   // is_last is rewritten by the next segment
+            for (int k = 0; k < kMaxPer; ++k) {
+                const int q = lane * per + k;
+                cnt[k] = (k < per && q < ngroups32) ? __popc(sm.group_mask[q]) : 0u;
+                mine += cnt[k];
+                if (q < qB) beforeB += cnt[k];
             }
+            beforeB = __reduce_add_sync(0xFFFFFFFFu, beforeB);         // records of piece A
+            const unsigned pad = (ngtB > 0) ? (kGroup - beforeB % kGroup) % kGroup : 0u;
+            if (ngtB > 0 && qB / per == lane) mine += pad;
+            unsigned inc = mine;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                unsigned v = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+                if (lane >= d) inc += v;
+            }
+            unsigned run = inc - mine;
+#pragma unroll
+            for (int k = 0; k < kMaxPer; ++k) {
+                const int q = lane * per + k;
+                if (k < per && q < ngroups32) {
+                    sm.group_base[q] = run;
+                    run += cnt[k] + ((ngtB > 0 && q == qB) ? pad : 0u);
+                }
+            }
+            if (lane == 31) sm.group_base[ngroups32] = inc;
+        }
+        __syncthreads();
+        const int nact = static_cast<int>(sm.group_base[ngroups32]);
+        const int ngroups = (nact + kGroup - 1) / kGroup;
+        // records of piece A end where piece B's first group starts (all of them if there is no piece B)
+        const int nactA_pad = (ngtB > 0) ? static_cast<int>(sm.group_base[qB] + (sm.group_base[qB + 1] - sm.group_base[qB] -
+                                                            __popc(sm.group_mask[qB])))
+                                         : ngroups * kGroup;
+        {
+            const int64_t slotA0 = gA * kTileK - jA0, slotB0 = gB * kTileK;          // column slot of column 0
+#pragma unroll 4
+            for (int q = warp; q < ngroups32; q += kWarps) {
+                const unsigned m = sm.group_mask[q];
+                if ((m >> lane) & 1u) {
+                    const int v = q * 32 + lane;
+                    const int j = (v < vB0) ? jA0 + v : v - vB0;
+                    const unsigned slot = static_cast<unsigned>((v < vB0 ? slotA0 : slotB0) + j);
+                    int item = static_cast<int>(sm.group_base[q] + __popc(m & ((1u << lane) - 1u)));
+                    if (q == qB) item += static_cast<int>(sm.group_base[qB + 1] - sm.group_base[qB]) - __popc(m);
+                    const uint32_t ci = sm.stage.colinfo[v];                        // ColInfo: offset << 16 | nnz
+                    sm.rec[item] = make_uint2(sm.stage.tileoff[v >> 4] + (ci >> 16), (slot << 6) | (((ci & 0xFFFFu) + 7u) >> 3));
+                    sm.xact[item] = sm.stage.x[v];
+                }
+            }
+            // null records: the padding in front of piece B and behind the last record
+            if (t < kGroup) {
+                const int padA = nactA_pad - t - 1;                 // the (up to kGroup-1) records before piece B
+                if (ngtB > 0 && t < kGroup - 1 && padA >= 0) {
+                    const int realA = static_cast<int>(sm.group_base[qB]);
+                    if (padA >= realA) sm.rec[padA] = make_uint2(0u, kNullRec);
+                }
+                sm.rec[nact + t] = make_uint2(0u, kNullRec);
+            }
+        }
+        __syncthreads();       // the records are complete; the staging area becomes the ring again
+
+        // ---- (2) per-warp fetch / decode pipeline over groups warp, warp + kWarps, ... ----
+        const int groupsA = nactA_pad / kGroup;                 // groups [0, groupsA) belong to piece A
+        // fetch(i): start the copies of my i-th group into ring position i % kDepth
+        auto fetch = [&](int i) {
+            const int lq = warp + i * kWarps;
+            if (lq < ngroups) {
+                const int d = i % kDepth;
+                const uint2 rc = lds_v2(rec_addr + 8u * (lq * kGroup + lgrp));
+                const uint32_t bdst = bm_own + d * 128;
+                if (rc.y != kNullRec) {
+                    const int rem = static_cast<int>(rc.y & 63u) - lane7;                  // my 16-byte pieces left
+                    const unsigned char* src = val_src + 2 * static_cast<uint64_t>(rc.x);
+                    const uint32_t dst = val_dst + d * kStageBytes;
+                    cp_async16<0>(dst, src, rem);
+                    cp_async16<128>(dst, src, rem);
+                    cp_async16<256>(dst, src, rem);
+                    cp_async16<384>(dst, src, rem);
+                    cp_async4(bdst, bm_src + static_cast<size_t>(rc.y >> 6) * 32);
+                } else {
+                    sts_u32(bdst, 0u);
+                }
+            }
+            cp_async_commit();
+        };
+#pragma unroll
+        for (int d = 0; d < kDepth; ++d) fetch(d);
+
+        int d = 0;
+        bool in_first = (ngtB > 0);                             // still inside piece A of a two-piece batch
+        for (int i = 0, lq = warp; lq < ngroups; ++i, lq += kWarps) {
+            if (in_first && lq >= groupsA) {
+                // my share of piece A is complete: park it and start piece B's row tile from zero
+                in_first = false;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    sm.red_first[warp][4 * lane + k] = acc[k];
+                    sm.red_first[warp][128 + 4 * lane + k] = acc[4 + k];
+                    acc[k] = 0.f;
+                    acc[4 + k] = 0.f;
+                }
+            }
+            cp_async_wait<kDepth - 1>();
+            __syncwarp();
+            // scan role: shared address of my word's first value
+            {
+                const unsigned cnt = __popc(lds_u32(bm_own + d * 128));
+                unsigned inc = cnt;
+#pragma unroll
+                for (int dd = 1; dd < 8; dd <<= 1) {
+                    unsigned v = __shfl_up_sync(0xFFFFFFFFu, inc, dd, 8);
+                    if (lane7 >= dd) inc += v;
+                }
+                sts_u32(va_own, slot_own + d * kStageBytes + 2u * (inc - cnt));
+            }
+            __syncwarp();
+            // decode role: my 8 words (tile it, word 4h + lgrp at index 2*it + h), their value addresses, the 4 x
+            const unsigned m1 = bit0 << 1, m2 = bit0 << 2, m3 = bit0 << 3;
+#pragma unroll 1
+            for (int half = 0; half < 2; ++half) {
+                const uint4 w = lds_v4(bm_dec + d * 128 + 16 * half);
+                const uint4 a = lds_v4(va_dec + 16 * half);
+                const unsigned xs = lds_u32(x_addr + 8u * lq + 4 * half);        // two activations
+                decode_step(w.x, a.x, lt_mask, bit0, m1, m2, m3, xs, acc[0], acc[1], acc[2], acc[3]);
+                decode_step(w.y, a.y, lt_mask, bit0, m1, m2, m3, xs, acc[4], acc[5], acc[6], acc[7]);
+                decode_step(w.z, a.z, lt_mask, bit0, m1, m2, m3, xs >> 16, acc[0], acc[1], acc[2], acc[3]);
+                decode_step(w.w, a.w, lt_mask, bit0, m1, m2, m3, xs >> 16, acc[4], acc[5], acc[6], acc[7]);
+            }
+            __syncwarp();                  // everyone is done with ring position d
+            fetch(i + kDepth);
+            d = (d + 1 == kDepth) ? 0 : d + 1;
+        }
+        if (in_first) {                    // this warp had no group of piece B: its piece-A sums are still in registers
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                sm.red_first[warp][4 * lane + k] = acc[k];
+                sm.red_first[warp][128 + 4 * lane + k] = acc[4 + k];
+                acc[k] = 0.f;
+                acc[4 + k] = 0.f;
+            }
+        }
+        cp_async_wait<0>();
+        __syncthreads();       // all pipelines drained: the ring is idle
+
+        // ---- (3) finish the row tiles this batch completed ----
+        const bool two = (ngtB > 0);
+        const bool done_last = two ? doneB : doneA;             // does the batch's last piece end its row tile here?
+        if (done_last) {
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                sm.red[warp][4 * lane + k] = acc[k];            // red[] reuses the idle ring
+                sm.red[warp][128 + 4 * lane + k] = acc[4 + k];
+                acc[k] = 0.f;
+                acc[4 + k] = 0.f;
+            }
+        }
+        __syncthreads();
+        // Threads 0..255 take the batch's last row tile, threads 256..511 the first one of a two-piece
+        // batch; the other warps go straight on to the next batch's list phase.  Neither red[] nor
+        // red_first[] is written again before these threads have passed the next __syncthreads.
+        if (t < kTileM) {
+            if (done_last) finish_row_tile(p, two ? rB : rA, r_first, sm.red, t, 1, &sm.is_last[0]);
+        } else if (t < 2 * kTileM) {
+            if (two) finish_row_tile(p, rA, r_first, sm.red_first, t - kTileM, 2, &sm.is_last[1]);
         }
     }
 }
@@ -532,7 +634,7 @@ spdp_status launch_spmspv_noalloc(const uint32_t* tileoffset, const uint32_t* co
     static int sm_count_of[kMaxDevices] = {};
     static std::mutex mu;
     const int64_t R = (M + kTileM - 1) / kTileM, C = (K + kTileK - 1) / kTileK, NGT = R * C;
-    if (R > kNoAllocMaxRowTiles || NGT >= (int64_t(1) << 31) / kTileK) return SPDP_ERR_UNSUPPORTED_SHAPE;
+    if (R > kNoAllocMaxRowTiles || NGT * kTileK >= (int64_t(1) << 26)) return SPDP_ERR_UNSUPPORTED_SHAPE;
     int dev = 0;
     SPDP_CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= kMaxDevices) return SPDP_ERR_UNSUPPORTED_SHAPE;

@@ -182,7 +182,8 @@ SPDP_API spdp_status spdp_active_columns(spdp_handle h, const void* x_dev, spdp_
  * Synchronises the device. */
 SPDP_API spdp_status spdp_last_device_status(spdp_handle h, int* out);
 
-/* Tuning knob: number of CTAs spdp_spmspv launches (0 = default, one per SM).  Takes effect on
+/* Tuning knob: number of CTAs spdp_spmspv launches (0 = default, one per SM; at most 1024 and at
+ * most one per GTile are used).  Takes effect on
  * the next call; re-derives the handle's split-K workspace layout (may reallocate it). */
 SPDP_API spdp_status spdp_set_num_ctas(spdp_handle h, int num_ctas);
 

@@ -4,7 +4,6 @@
 #include <cstdio>
 #include <cstring>
 #include <new>
-#include <vector>
 
 #include "spdp_internal.h"
 
@@ -26,9 +25,6 @@ void release(spdp_matrix* h) {
     cudaFree(h->colinfo);
     cudaFree(h->bitmap);
     cudaFree(h->values);
-    cudaFree(h->cta_begin);
-    cudaFree(h->row_first_cta);
-    cudaFree(h->row_nseg);
     cudaFree(h->workspace);
     cudaFree(h->row_counter);
     cudaFree(h->status_word);
@@ -61,38 +57,20 @@ spdp_status new_handle(int64_t M, int64_t K, int pad_elems, spdp_matrix** out) {
     return SPDP_OK;
 }
 
-// Cuts the NGT GTiles into num_ctas equal contiguous ranges and derives, per row tile, which
-// CTAs feed it.  (Re)allocates the tables, the workspace and the counters.
+// Chooses the number of CTAs (the kernel cuts the NGT GTiles into that many equal contiguous
+// ranges) and (re)allocates what depends on it: the split-K workspace and the arrival counters.
 spdp_status build_partition(spdp_matrix* h, int num_ctas) {
-    const int64_t NGT = h->NGT, C = h->C, R = h->R;
+    const int64_t NGT = h->NGT, R = h->R;
     int P = num_ctas > 0 ? num_ctas : h->sm_count * default_ctas_per_sm();
+    if (P > 1024) P = 1024;          // the kernel's range arithmetic is 32-bit: NGT < 2^22 times P must fit
     if (P > NGT) P = static_cast<int>(NGT);
     if (P < 1) P = 1;
-    std::vector<uint32_t> begin(P + 1);
-    for (int p = 0; p <= P; ++p) begin[p] = static_cast<uint32_t>((static_cast<__int128>(NGT) * p) / P);
-    std::vector<int32_t> first(R, -1), nseg(R, 0);
-    for (int p = 0; p < P; ++p) {
-        const int64_t r0 = begin[p] / C, r1 = (static_cast<int64_t>(begin[p + 1]) - 1) / C;
-        for (int64_t r = r0; r <= r1; ++r) {
-            if (first[r] < 0) first[r] = p;
-            ++nseg[r];
-        }
-    }
-    cudaFree(h->cta_begin);     h->cta_begin = nullptr;
-    cudaFree(h->row_first_cta); h->row_first_cta = nullptr;
-    cudaFree(h->row_nseg);      h->row_nseg = nullptr;
     cudaFree(h->workspace);     h->workspace = nullptr;
     cudaFree(h->row_counter);   h->row_counter = nullptr;
     h->num_ctas = P;
     h->workspace_bytes = static_cast<int64_t>(P) * 2 * kTileM * sizeof(float);   // two slots per CTA
-    SPDP_CUDA_TRY(cudaMalloc(&h->cta_begin, (P + 1) * sizeof(uint32_t)));
-    SPDP_CUDA_TRY(cudaMalloc(&h->row_first_cta, R * sizeof(int32_t)));
-    SPDP_CUDA_TRY(cudaMalloc(&h->row_nseg, R * sizeof(int32_t)));
     SPDP_CUDA_TRY(cudaMalloc(&h->workspace, h->workspace_bytes));
     SPDP_CUDA_TRY(cudaMalloc(&h->row_counter, R * sizeof(unsigned)));
-    SPDP_CUDA_TRY(cudaMemcpy(h->cta_begin, begin.data(), (P + 1) * sizeof(uint32_t), cudaMemcpyHostToDevice));
-    SPDP_CUDA_TRY(cudaMemcpy(h->row_first_cta, first.data(), R * sizeof(int32_t), cudaMemcpyHostToDevice));
-    SPDP_CUDA_TRY(cudaMemcpy(h->row_nseg, nseg.data(), R * sizeof(int32_t), cudaMemcpyHostToDevice));
     SPDP_CUDA_TRY(cudaMemset(h->workspace, 0, h->workspace_bytes));
     SPDP_CUDA_TRY(cudaMemset(h->row_counter, 0, R * sizeof(unsigned)));
     return SPDP_OK;

@@ -32,11 +32,9 @@ struct spdp_matrix {
     uint64_t* bitmap;       // [NGT*16*4]
     __half* values;         // [values_len] (at least 16 bytes are allocated)
 
-    // Work partition of one spmspv launch: CTA p owns GTiles [cta_begin[p], cta_begin[p+1]).
+    // Work partition of one spmspv launch: the kernel cuts the NGT GTiles into num_ctas equal
+    // contiguous ranges, one per CTA.
     int num_ctas;           // P
-    uint32_t* cta_begin;    // device [P+1]
-    int32_t* row_first_cta; // device [R]: first CTA whose range touches row tile r
-    int32_t* row_nseg;      // device [R]: number of CTAs whose range touches row tile r
     float* workspace;       // device [P*2*256] split-K partial sums (two slots per CTA)
     unsigned* row_counter;  // device [R] arrivals per row tile (self-resetting)
     int* status_word;       // device [1]

@@ -43,6 +43,7 @@ constexpr int kThreads = kWarps * 32;
 constexpr int kChunkCols = SPDP_CHUNK_COLS; // columns handled between two pipeline drains
 constexpr int kCtasPerSm = SPDP_CTAS_PER_SM;
 constexpr uint32_t kNullRec = 0xFFFFFFFFu;
+constexpr int kMaxGroupsPerWarp = (kChunkCols / 32 + kWarps - 1) / kWarps;   // 32-position groups a warp lists per batch
 constexpr int kChunkGT = kChunkCols / kTileK;
 
 struct Params {
@@ -57,9 +58,8 @@ struct Params {
     int rule;
     int ydt;
     int M, K, R, C;
-    const uint32_t* cta_begin;
-    const int32_t* row_first_cta;
-    const int32_t* row_nseg;
+    int64_t NGT;            // R * C GTiles, cut into num_ctas equal contiguous ranges
+    int num_ctas;
     float* workspace;
     unsigned* row_counter;
     int* status;
@@ -86,8 +86,7 @@ struct __align__(128) Smem {
                                                         //      of values; kNullRec pads a piece to whole groups
     alignas(16) unsigned short xact[kChunkCols + kGroup];   // its activation x_j (fp16 bits)
     float red_first[kWarps][kTileM];                    // row reduction of a batch's first piece (flushed mid-stream)
-    uint32_t group_mask[kChunkCols / 32];
-    uint32_t group_base[kChunkCols / 32 + 1];
+    uint32_t warp_total[kWarps][2];                     // list phase: records listed by each warp (all, piece A)
     int is_last[2];
 };
 static_assert(offsetof(Smem, rec) % 16 == 0 && offsetof(Smem, xact) % 16 == 0 && offsetof(Smem, vaddr) % 16 == 0 &&
@@ -194,6 +193,17 @@ __device__ __forceinline__ void sts_u32(uint32_t addr, unsigned v) {
     asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
 
+// The work split: CTA c owns GTiles [range_begin(c), range_begin(c + 1)) of the row-major GTile order.
+// NGT < 2^22 and num_ctas <= 1024 keep every product below 2^32.
+__device__ __forceinline__ unsigned range_begin(const Params& p, unsigned c) {
+    return (static_cast<unsigned>(p.NGT) * c) / static_cast<unsigned>(p.num_ctas);
+}
+// The CTA whose range holds GTile g: ceil((g + 1) * num_ctas / NGT) - 1.
+__device__ __forceinline__ int range_owner(const Params& p, unsigned g) {
+    const unsigned ngt = static_cast<unsigned>(p.NGT);
+    return static_cast<int>(((g + 1u) * static_cast<unsigned>(p.num_ctas) + ngt - 1u) / ngt) - 1;
+}
+
 // Adds the kWarps per-warp partial sums of one row tile in warp order and finishes the row tile
 // (256 threads, tt = row inside the tile, `bar` = a named barrier of these 256 threads).  A row tile
 // fed by one segment is stored directly; otherwise the sum goes to this CTA's workspace slot and
@@ -204,27 +214,29 @@ __device__ __forceinline__ void finish_row_tile(const Params& p, int r, int r_fi
 #pragma unroll
     for (int w = 0; w < kWarps; ++w) part += red[w][tt];
     const int64_t row = static_cast<int64_t>(r) * kTileM + tt;
-    const int nseg = p.row_nseg[r];
+    const int q0 = range_owner(p, static_cast<unsigned>(r) * p.C);                 // first and last CTA feeding row tile r
+    const int nseg = range_owner(p, static_cast<unsigned>(r + 1) * p.C - 1u) - q0 + 1;
     if (nseg == 1) {
         if (row < p.M) store_y(p.y, p.ydt, row, part);
         return;
     }
     __stcg(p.workspace + (static_cast<int64_t>(blockIdx.x) * 2 + (r != r_first)) * kTileM + tt, part);
-    __threadfence();
+    // The barrier orders the 256 partial sums before thread 0's acq_rel arrival (release: they are
+    // visible to whoever sees the count; acquire: it sees the partials of every earlier arrival), and
+    // the second barrier hands that view to the other 255 threads.
     asm volatile("bar.sync %0, 256;" ::"r"(bar) : "memory");
     if (tt == 0) {
-        const unsigned old = atomicAdd(p.row_counter + r, 1u);
+        unsigned old;
+        asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(p.row_counter + r) : "memory");
         *is_last = (old == static_cast<unsigned>(nseg - 1));
     }
     asm volatile("bar.sync %0, 256;" ::"r"(bar) : "memory");
     if (*is_last) {
-        __threadfence();
         if (row < p.M) {
-            const int q0 = p.row_first_cta[r];
             float sum = 0.f;
             for (int s = 0; s < nseg; ++s) {
                 const int q = q0 + s;
-                const int slot = (r != static_cast<int>(p.cta_begin[q] / p.C));
+                const int slot = (r != static_cast<int>(range_begin(p, q) / static_cast<unsigned>(p.C)));
                 sum += __ldcg(p.workspace + (static_cast<int64_t>(q) * 2 + slot) * kTileM + tt);
             }
             store_y(p.y, p.ydt, row, sum);
@@ -256,8 +268,8 @@ spmspv_kernel(const Params p) {
     Smem& sm = *reinterpret_cast<Smem*>(smem_raw);
 
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
-    const int64_t g_begin = p.cta_begin[blockIdx.x], g_end = p.cta_begin[blockIdx.x + 1];
-    const int r_first = static_cast<int>(g_begin / p.C);
+    const int64_t g_begin = range_begin(p, blockIdx.x), g_end = range_begin(p, blockIdx.x + 1);
+    const int r_first = static_cast<int>(static_cast<unsigned>(g_begin) / static_cast<unsigned>(p.C));
 
     const int lane7 = lane & 7;
     const int lgrp = lane >> 3;
@@ -284,7 +296,7 @@ spmspv_kernel(const Params p) {
 
     for (int64_t g0 = g_begin; g0 < g_end;) {
         // ---- the batch: piece A = [gA, gA + ngtA) of row tile rA, optionally piece B of row tile rA + 1 ----
-        const int rA = static_cast<int>(g0 / p.C);
+        const int rA = static_cast<int>(static_cast<unsigned>(g0) / static_cast<unsigned>(p.C));
         const int cA = static_cast<int>(g0 - static_cast<int64_t>(rA) * p.C);
         int ngtA = p.C - cA;
         if (ngtA > g_end - g0) ngtA = static_cast<int>(g_end - g0);
@@ -339,89 +351,71 @@ spmspv_kernel(const Params p) {
         }
         cp_async_wait<0>();
         __syncthreads();
-#pragma unroll 4
-        for (int q = warp; q < ngroups32; q += kWarps) {
-            const int v = q * 32 + lane;                             // list position
-            const int j = (v < vB0) ? jA0 + v : v - vB0;             // its column
-            bool a = (v < vB0) ? (v < nA) : (v < nlist);
-            if (a) {
-                if (p.rule == SPDP_DP_ABS_GT)
-                    a = !(fabsf(__half2float(__ushort_as_half(sm.stage.x[v]))) <= p.thr);
-                else if (p.rule == SPDP_DP_MASK)
-                    a = (__ldg(p.mask + (j >> 5)) >> (j & 31)) & 1u;
-            }
-            const unsigned m = __ballot_sync(0xFFFFFFFFu, a);
-            if (lane == 0) sm.group_mask[q] = m;
-        }
-        __syncthreads();
-        if (warp == 0) {
-            // Exclusive prefix sums of the group counts: lane l owns groups [l*per, (l+1)*per).  Piece B
-            // starts on a whole group of kGroup records: the padding is counted in front of its first group.
-            constexpr int kMaxPer = (kChunkCols / 32 + 31) / 32;
-            const int per = (ngroups32 + 31) >> 5;
-            unsigned cnt[kMaxPer];
-            unsigned mine = 0, beforeB = 0;
-#pragma unroll
-            for (int k = 0; k < kMaxPer; ++k) {
-                const int q = lane * per + k;
-                cnt[k] = (k < per && q < ngroups32) ? __popc(sm.group_mask[q]) : 0u;
-                mine += cnt[k];
-                if (q < qB) beforeB += cnt[k];
-            }
-            beforeB = __reduce_add_sync(0xFFFFFFFFu, beforeB);         // records of piece A
-            const unsigned pad = (ngtB > 0) ? (kGroup - beforeB % kGroup) % kGroup : 0u;
-            if (ngtB > 0 && qB / per == lane) mine += pad;
-            unsigned inc = mine;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                unsigned v = __shfl_up_sync(0xFFFFFFFFu, inc, d);
-                if (lane >= d) inc += v;
-            }
-            unsigned run = inc - mine;
-#pragma unroll
-            for (int k = 0; k < kMaxPer; ++k) {
-                const int q = lane * per + k;
-                if (k < per && q < ngroups32) {
-                    sm.group_base[q] = run;
-                    run += cnt[k] + ((ngtB > 0 && q == qB) ? pad : 0u);
-                }
-            }
-            if (lane == 31) sm.group_base[ngroups32] = inc;
-        }
-        __syncthreads();
-        const int nact = static_cast<int>(sm.group_base[ngroups32]);
-        const int ngroups = (nact + kGroup - 1) / kGroup;
-        // records of piece A end where piece B's first group starts (all of them if there is no piece B)
-        const int nactA_pad = (ngtB > 0) ? static_cast<int>(sm.group_base[qB] + (sm.group_base[qB + 1] - sm.group_base[qB] -
-                                                            __popc(sm.group_mask[qB])))
-                                         : ngroups * kGroup;
+        // Warp w lists the 32-position groups [w * gpw, (w + 1) * gpw): one ballot per group, kept in
+        // registers; the warps' totals meet in shared memory, every warp derives its first record index
+        // from them, and the records are written in list order.  Piece B starts on a whole group of
+        // kGroup records: the padding is inserted in front of its first record.
+        const int gpw = (ngroups32 + kWarps - 1) / kWarps;
+        unsigned masks[kMaxGroupsPerWarp];
         {
-            const int64_t slotA0 = gA * kTileK - jA0, slotB0 = gB * kTileK;          // column slot of column 0
-#pragma unroll 4
-            for (int q = warp; q < ngroups32; q += kWarps) {
-                const unsigned m = sm.group_mask[q];
+            unsigned tot = 0, totA = 0;
+#pragma unroll
+            for (int k = 0; k < kMaxGroupsPerWarp; ++k) {
+                const int q = warp * gpw + k;
+                const int v = q * 32 + lane;                             // list position
+                const int j = (v < vB0) ? jA0 + v : v - vB0;             // its column
+                bool a = (k < gpw) && ((v < vB0) ? (v < nA) : (v < nlist));
+                if (a) {
+                    if (p.rule == SPDP_DP_ABS_GT)
+                        a = !(fabsf(__half2float(__ushort_as_half(sm.stage.x[v]))) <= p.thr);
+                    else if (p.rule == SPDP_DP_MASK)
+                        a = (__ldg(p.mask + (j >> 5)) >> (j & 31)) & 1u;
+                }
+                masks[k] = __ballot_sync(0xFFFFFFFFu, a);
+                const unsigned c = __popc(masks[k]);
+                tot += c;
+                if (q < qB) totA += c;
+            }
+            if (lane == 0) {
+                sm.warp_total[warp][0] = tot;
+                sm.warp_total[warp][1] = totA;
+            }
+        }
+        __syncthreads();
+        int nact, nactA_pad;
+        {
+            const unsigned tl = (lane < kWarps) ? sm.warp_total[lane][0] : 0u;
+            const unsigned tla = (lane < kWarps) ? sm.warp_total[lane][1] : 0u;
+            const unsigned realA = __reduce_add_sync(0xFFFFFFFFu, tla);                     // records of piece A
+            const unsigned pad = (ngtB > 0) ? (kGroup - realA % kGroup) % kGroup : 0u;
+            const unsigned total = __reduce_add_sync(0xFFFFFFFFu, tl) + pad;
+            unsigned base = __reduce_add_sync(0xFFFFFFFFu, lane < warp ? tl : 0u);          // before my first group
+            nact = static_cast<int>(total);
+            nactA_pad = (ngtB > 0) ? static_cast<int>(realA + pad) : ((nact + kGroup - 1) / kGroup) * kGroup;
+            const int64_t slotA0 = gA * kTileK - jA0, slotB0 = gB * kTileK;                  // column slot of column 0
+#pragma unroll
+            for (int k = 0; k < kMaxGroupsPerWarp; ++k) {
+                const int q = warp * gpw + k;
+                const unsigned m = masks[k];
                 if ((m >> lane) & 1u) {
                     const int v = q * 32 + lane;
                     const int j = (v < vB0) ? jA0 + v : v - vB0;
                     const unsigned slot = static_cast<unsigned>((v < vB0 ? slotA0 : slotB0) + j);
-                    int item = static_cast<int>(sm.group_base[q] + __popc(m & ((1u << lane) - 1u)));
-                    if (q == qB) item += static_cast<int>(sm.group_base[qB + 1] - sm.group_base[qB]) - __popc(m);
-                    const uint32_t ci = sm.stage.colinfo[v];                        // ColInfo: offset << 16 | nnz
+                    const int item = static_cast<int>(base + (q >= qB ? pad : 0u) + __popc(m & ((1u << lane) - 1u)));
+                    const uint32_t ci = sm.stage.colinfo[v];                                // ColInfo: offset << 16 | nnz
                     sm.rec[item] = make_uint2(sm.stage.tileoff[v >> 4] + (ci >> 16), (slot << 6) | (((ci & 0xFFFFu) + 7u) >> 3));
                     sm.xact[item] = sm.stage.x[v];
                 }
+                base += __popc(m);
             }
             // null records: the padding in front of piece B and behind the last record
-            if (t < kGroup) {
-                const int padA = nactA_pad - t - 1;                 // the (up to kGroup-1) records before piece B
-                if (ngtB > 0 && t < kGroup - 1 && padA >= 0) {
-                    const int realA = static_cast<int>(sm.group_base[qB]);
-                    if (padA >= realA) sm.rec[padA] = make_uint2(0u, kNullRec);
-                }
-                sm.rec[nact + t] = make_uint2(0u, kNullRec);
+            if (warp == 0) {
+                if (lane < static_cast<int>(pad)) sm.rec[realA + lane] = make_uint2(0u, kNullRec);
+                if (lane < kGroup) sm.rec[nact + lane] = make_uint2(0u, kNullRec);
             }
         }
         __syncthreads();       // the records are complete; the staging area becomes the ring again
+        const int ngroups = (nact + kGroup - 1) / kGroup;
 
         // ---- (2) per-warp fetch / decode pipeline over groups warp, warp + kWarps, ... ----
         const int groupsA = nactA_pad / kGroup;                 // groups [0, groupsA) belong to piece A
@@ -569,9 +563,6 @@ constexpr int kNoAllocMaxCtas = 512;
 constexpr int kNoAllocMaxRowTiles = 4096;          // M <= 1,048,576
 
 struct NoAllocScratch {
-    uint32_t cta_begin[kNoAllocMaxCtas + 1];
-    int32_t row_first_cta[kNoAllocMaxRowTiles];
-    int32_t row_nseg[kNoAllocMaxRowTiles];
     unsigned row_counter[kNoAllocMaxRowTiles];
     int status;
     float workspace[kNoAllocMaxCtas * 2 * kTileM];
@@ -579,21 +570,10 @@ struct NoAllocScratch {
 
 static __device__ __align__(256) unsigned char g_noalloc_scratch[sizeof(NoAllocScratch)];
 
-// Fills the partition tables for P CTAs and zeroes what a call expects to start at zero (the
-// array keeps whatever the previous call left).
-__global__ void noalloc_setup_kernel(NoAllocScratch* sc, int64_t NGT, int64_t C, int R, int P) {
-    for (int p = threadIdx.x; p <= P; p += blockDim.x)
-        sc->cta_begin[p] = static_cast<uint32_t>((static_cast<unsigned long long>(NGT) * p) / P);
-    for (int r = threadIdx.x; r < R; r += blockDim.x) {
-        // the CTA whose range holds GTile s is ceil((s+1)*P/NGT) - 1
-        const unsigned long long s0 = static_cast<unsigned long long>(r) * C, s1 = s0 + C - 1;
-        const int first = static_cast<int>(((s0 + 1) * P + NGT - 1) / NGT) - 1;
-        const int last = static_cast<int>(((s1 + 1) * P + NGT - 1) / NGT) - 1;
-        sc->row_first_cta[r] = first;
-        sc->row_nseg[r] = last - first + 1;
-        sc->row_counter[r] = 0;
-    }
-    if (threadIdx.x == 0) sc->status = 0;
+// Zeroes what a call expects to start at zero (the array keeps whatever the previous call left).
+__global__ void noalloc_setup_kernel(NoAllocScratch* sc, int R) {
+    for (int r = blockIdx.x * blockDim.x + threadIdx.x; r < R; r += gridDim.x * blockDim.x) sc->row_counter[r] = 0;
+    if (blockIdx.x == 0 && threadIdx.x == 0) sc->status = 0;
 }
 
 }  // namespace
@@ -617,9 +597,8 @@ spdp_status launch_spmspv(const spdp_matrix* h, const __half* x, int rule, float
     p.K = static_cast<int>(h->K);
     p.R = static_cast<int>(h->R);
     p.C = static_cast<int>(h->C);
-    p.cta_begin = h->cta_begin;
-    p.row_first_cta = h->row_first_cta;
-    p.row_nseg = h->row_nseg;
+    p.NGT = h->NGT;
+    p.num_ctas = h->num_ctas;
     p.workspace = h->workspace;
     p.row_counter = h->row_counter;
     p.status = h->status_word;
@@ -655,7 +634,7 @@ spdp_status launch_spmspv_noalloc(const uint32_t* tileoffset, const uint32_t* co
     }
     int P = sms * kCtasPerSm < kNoAllocMaxCtas ? sms * kCtasPerSm : kNoAllocMaxCtas;
     if (P > NGT) P = static_cast<int>(NGT);
-    noalloc_setup_kernel<<<1, 256, 0, s>>>(sc, NGT, C, static_cast<int>(R), P);
+    noalloc_setup_kernel<<<(static_cast<int>(R) + 255) / 256, 256, 0, s>>>(sc, static_cast<int>(R));
     SPDP_CUDA_TRY(cudaGetLastError());
     Params p;
     p.tileoffset = tileoffset;
@@ -672,10 +651,9 @@ spdp_status launch_spmspv_noalloc(const uint32_t* tileoffset, const uint32_t* co
     p.K = static_cast<int>(K);
     p.R = static_cast<int>(R);
     p.C = static_cast<int>(C);
-    p.cta_begin = sc->cta_begin;            // addresses inside the device array (no host dereference)
-    p.row_first_cta = sc->row_first_cta;
-    p.row_nseg = sc->row_nseg;
-    p.workspace = sc->workspace;
+    p.NGT = NGT;
+    p.num_ctas = P;
+    p.workspace = sc->workspace;            // addresses inside the device array (no host dereference)
     p.row_counter = sc->row_counter;
     p.status = &sc->status;
     return launch_kernel(p, P, s);

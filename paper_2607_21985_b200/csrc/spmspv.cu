@@ -79,7 +79,7 @@ struct __align__(128) Smem {
     // Bitmap words of a group in decode order: word w of the group's it-th tile sits at
     // [(w & 3) * 8 + it * 2 + (w >> 2)], so the lanes that decode words (w & 3) == g read 8 consecutive words.
     alignas(16) uint32_t bmring[kWarps][kDepth][32];
-    alignas(16) uint32_t vaddr[kWarps][32];             // same order: shared address of each word's first value
+    alignas(16) unsigned short voff[kWarps][32];        // same order: byte offset of each word's first value in the warp's ring
     // Active list of the chunk, one record per active column tile (filled once per chunk):
     alignas(16) uint2 rec[kChunkCols + kGroup];         // .x = start of its values in Values (elements),
                                                         // .y = (column slot in Bitmap/ColInfo) << 6 | 16-byte pieces
@@ -89,7 +89,7 @@ struct __align__(128) Smem {
     uint32_t warp_total[kWarps][2];                     // list phase: records listed by each warp (all, piece A)
     int is_last[2];
 };
-static_assert(offsetof(Smem, rec) % 16 == 0 && offsetof(Smem, xact) % 16 == 0 && offsetof(Smem, vaddr) % 16 == 0 &&
+static_assert(offsetof(Smem, rec) % 16 == 0 && offsetof(Smem, xact) % 16 == 0 && offsetof(Smem, voff) % 16 == 0 &&
               offsetof(Smem, bmring) % 16 == 0, "16-byte shared loads need aligned tables");
 static_assert(sizeof(float) * kWarps * kTileM <= size_t(kWarps) * kDepth * kStageBytes, "red must fit in the ring");
 static_assert(sizeof(uint32_t) * (kChunkCols + kChunkGT) + 2 * kChunkCols + sizeof(float) * kWarps * kTileM <=
@@ -189,6 +189,9 @@ __device__ __forceinline__ uint2 lds_v2(uint32_t addr) {
     asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
     return v;
 }
+__device__ __forceinline__ void sts_u16(uint32_t addr, unsigned v) {
+    asm volatile("{\n .reg .b16 h;\n cvt.u16.u32 h, %1;\n st.shared.u16 [%0], h;\n}" ::"r"(addr), "r"(v) : "memory");
+}
 __device__ __forceinline__ void sts_u32(uint32_t addr, unsigned v) {
     asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
@@ -282,9 +285,9 @@ spmspv_kernel(const Params p) {
     const uint32_t val_dst = smem_u32(&sm.ring[warp][0][lgrp * kSlotBytes + 16 * lane7]);
     const uint32_t bm_own = smem_u32(&sm.bmring[warp][0][tpos]);
     const uint32_t bm_dec = smem_u32(&sm.bmring[warp][0][lgrp * 8]);
-    const uint32_t va_own = smem_u32(&sm.vaddr[warp][tpos]);
-    const uint32_t va_dec = smem_u32(&sm.vaddr[warp][lgrp * 8]);
-    const uint32_t slot_own = smem_u32(&sm.ring[warp][0][lgrp * kSlotBytes]);      // scan role: my tile's slot
+    const uint32_t vo_own = smem_u32(&sm.voff[warp][tpos]);
+    const uint32_t vo_dec = smem_u32(&sm.voff[warp][lgrp * 8]);
+    const uint32_t ring_w = smem_u32(&sm.ring[warp][0][0]);                         // my warp's ring
     const uint32_t rec_addr = smem_u32(&sm.rec[0]);
     const uint32_t x_addr = smem_u32(&sm.xact[0]);
     const unsigned char* bm_src = reinterpret_cast<const unsigned char*>(p.bitmap) + lane7 * 4;     // fetch role
@@ -469,7 +472,7 @@ spmspv_kernel(const Params p) {
                     unsigned v = __shfl_up_sync(0xFFFFFFFFu, inc, dd, 8);
                     if (lane7 >= dd) inc += v;
                 }
-                sts_u32(va_own, slot_own + d * kStageBytes + 2u * (inc - cnt));
+                sts_u16(vo_own, lgrp * kSlotBytes + d * kStageBytes + 2u * (inc - cnt));
             }
             __syncwarp();
             // decode role: my 8 words (tile it, word 4h + lgrp at index 2*it + h), their value addresses, the 4 x
@@ -477,12 +480,12 @@ spmspv_kernel(const Params p) {
 #pragma unroll 1
             for (int half = 0; half < 2; ++half) {
                 const uint4 w = lds_v4(bm_dec + d * 128 + 16 * half);
-                const uint4 a = lds_v4(va_dec + 16 * half);
+                const uint2 a = lds_v2(vo_dec + 8 * half);                       // four 16-bit offsets
                 const unsigned xs = lds_u32(x_addr + 8u * lq + 4 * half);        // two activations
-                decode_step(w.x, a.x, lt_mask, bit0, m1, m2, m3, xs, acc[0], acc[1], acc[2], acc[3]);
-                decode_step(w.y, a.y, lt_mask, bit0, m1, m2, m3, xs, acc[4], acc[5], acc[6], acc[7]);
-                decode_step(w.z, a.z, lt_mask, bit0, m1, m2, m3, xs >> 16, acc[0], acc[1], acc[2], acc[3]);
-                decode_step(w.w, a.w, lt_mask, bit0, m1, m2, m3, xs >> 16, acc[4], acc[5], acc[6], acc[7]);
+                decode_step(w.x, ring_w + (a.x & 0xFFFFu), lt_mask, bit0, m1, m2, m3, xs, acc[0], acc[1], acc[2], acc[3]);
+                decode_step(w.y, ring_w + (a.x >> 16), lt_mask, bit0, m1, m2, m3, xs, acc[4], acc[5], acc[6], acc[7]);
+                decode_step(w.z, ring_w + (a.y & 0xFFFFu), lt_mask, bit0, m1, m2, m3, xs >> 16, acc[0], acc[1], acc[2], acc[3]);
+                decode_step(w.w, ring_w + (a.y >> 16), lt_mask, bit0, m1, m2, m3, xs >> 16, acc[4], acc[5], acc[6], acc[7]);
             }
             __syncwarp();                  // everyone is done with ring position d
             fetch(i + kDepth);

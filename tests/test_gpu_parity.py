@@ -150,7 +150,9 @@ def test_active_set_bit_exact(S):
 @pytest.mark.parametrize("M,K,sp,skip,seed", [
     (256, 16, 0.5, 0.5, 1), (512, 64, 0.5, 0.0, 2), (300, 40, 0.3, 0.25, 3), (1, 1, 0.0, 0.0, 4),
     (257, 17, 0.5, 0.5, 5), (1024, 1024, 0.5, 0.5, 6), (768, 4400, 0.7, 0.9, 7), (2304, 528, 0.9, 0.4, 8),
-    (4096, 272, 0.0, 0.1, 9), (256, 8192, 0.6, 0.5, 10)])
+    (4096, 272, 0.0, 0.1, 9), (256, 8192, 0.6, 0.5, 10),
+    # rows longer than one batch of the kernel (pieces carry their sums over) and ragged long rows
+    (512, 20000, 0.5, 0.3, 11), (300, 16400, 0.9, 0.0, 12), (1000, 8200, 0.2, 0.6, 13)])
 @pytest.mark.parametrize("ydtype", ["f32", "f16"])
 def test_spmspv_matches_oracle(S, M, K, sp, skip, seed, ydtype):
     rw, rx = WL._rngs(seed)

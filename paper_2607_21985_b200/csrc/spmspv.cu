@@ -174,6 +174,12 @@ __device__ __forceinline__ void decode_step(unsigned W, uint32_t first, unsigned
         : "+f"(a0), "+f"(a1), "+f"(a2), "+f"(a3)
         : "r"(W), "r"(first), "r"(below), "r"(m0), "r"(m1), "r"(m2), "r"(m3), "r"(x32));
 }
+// One level of an inclusive prefix sum over segments of 8 lanes.
+template <int kDelta>
+__device__ __forceinline__ void scan8_level(unsigned& v) {
+    asm volatile("{\n .reg .pred p;\n .reg .b32 u;\n shfl.sync.up.b32 u|p, %0, %1, 0x1800, 0xffffffff;\n @p add.u32 %0, %0, u;\n}"
+                 : "+r"(v) : "n"(kDelta));
+}
 __device__ __forceinline__ unsigned lds_u32(uint32_t addr) {
     unsigned v;
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
@@ -271,8 +277,8 @@ spmspv_kernel(const Params p) {
     Smem& sm = *reinterpret_cast<Smem*>(smem_raw);
 
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
-    const int64_t g_begin = range_begin(p, blockIdx.x), g_end = range_begin(p, blockIdx.x + 1);
-    const int r_first = static_cast<int>(static_cast<unsigned>(g_begin) / static_cast<unsigned>(p.C));
+    const unsigned g_begin = range_begin(p, blockIdx.x), g_end = range_begin(p, blockIdx.x + 1);
+    const int r_first = static_cast<int>(g_begin / static_cast<unsigned>(p.C));
 
     const int lane7 = lane & 7;
     const int lgrp = lane >> 3;
@@ -288,23 +294,22 @@ spmspv_kernel(const Params p) {
     const uint32_t vo_own = smem_u32(&sm.voff[warp][tpos]);
     const uint32_t vo_dec = smem_u32(&sm.voff[warp][lgrp * 8]);
     const uint32_t ring_w = smem_u32(&sm.ring[warp][0][0]);                         // my warp's ring
+    const uint32_t slot_off = lgrp * kSlotBytes;                                    // scan role: my tile's slot in a stage
     const uint32_t rec_addr = smem_u32(&sm.rec[0]);
     const uint32_t x_addr = smem_u32(&sm.xact[0]);
-    const unsigned char* bm_src = reinterpret_cast<const unsigned char*>(p.bitmap) + lane7 * 4;     // fetch role
-    const unsigned char* val_src = reinterpret_cast<const unsigned char*>(p.values) + 16 * lane7;   // fetch role
 
     float acc[8];                   // rows 4*lane+k (k<4) and 128+4*lane+(k-4) of the current row tile
 #pragma unroll
     for (int k = 0; k < 8; ++k) acc[k] = 0.f;
 
-    for (int64_t g0 = g_begin; g0 < g_end;) {
+    for (unsigned g0 = g_begin; g0 < g_end;) {
         // ---- the batch: piece A = [gA, gA + ngtA) of row tile rA, optionally piece B of row tile rA + 1 ----
-        const int rA = static_cast<int>(static_cast<unsigned>(g0) / static_cast<unsigned>(p.C));
-        const int cA = static_cast<int>(g0 - static_cast<int64_t>(rA) * p.C);
+        const int rA = static_cast<int>(g0 / static_cast<unsigned>(p.C));
+        const int cA = static_cast<int>(g0 - static_cast<unsigned>(rA) * static_cast<unsigned>(p.C));
         int ngtA = p.C - cA;
-        if (ngtA > g_end - g0) ngtA = static_cast<int>(g_end - g0);
+        if (ngtA > static_cast<int>(g_end - g0)) ngtA = static_cast<int>(g_end - g0);
         if (ngtA > kChunkGT) ngtA = kChunkGT;
-        const int64_t gA = g0;
+        const unsigned gA = g0;
         g0 += ngtA;
         const bool doneA = (cA + ngtA == p.C) || (g0 == g_end);     // piece A ends its row tile's share of this CTA
         const int jA0 = cA * kTileK;
@@ -314,12 +319,12 @@ spmspv_kernel(const Params p) {
         bool doneB = false;
         if (doneA && g0 < g_end && cA + ngtA == p.C) {
             ngtB = p.C;
-            if (ngtB > g_end - g0) ngtB = static_cast<int>(g_end - g0);
+            if (ngtB > static_cast<int>(g_end - g0)) ngtB = static_cast<int>(g_end - g0);
             if (ngtB > (kChunkCols - vB0) / kTileK) ngtB = (kChunkCols - vB0) / kTileK;
             nB = min(ngtB * kTileK, p.K);
             doneB = (ngtB == p.C) || (g0 + ngtB == g_end);
         }
-        const int64_t gB = g0;
+        const unsigned gB = g0;
         g0 += ngtB;
         const int rB = rA + 1;
         const int nlist = (ngtB > 0) ? vB0 + nB : nA;               // list positions (A, padding, B)
@@ -334,8 +339,8 @@ spmspv_kernel(const Params p) {
             const uint32_t ci_stage = smem_u32(&sm.stage.colinfo[0]);
             const uint32_t to_stage = smem_u32(&sm.stage.tileoff[0]);
             const uint32_t x_stage = smem_u32(&sm.stage.x[0]);
-            const uint4* ciA = reinterpret_cast<const uint4*>(p.colinfo + gA * kTileK);
-            const uint4* ciB = reinterpret_cast<const uint4*>(p.colinfo + gB * kTileK);
+            const uint4* ciA = reinterpret_cast<const uint4*>(p.colinfo + static_cast<size_t>(gA) * kTileK);
+            const uint4* ciB = reinterpret_cast<const uint4*>(p.colinfo + static_cast<size_t>(gB) * kTileK);
             for (int i = t; i < ngtA * (kTileK / 4); i += kThreads) cp_async16<0>(ci_stage + 16 * i, ciA + i, 1);
             for (int i = t; i < ngtB * (kTileK / 4); i += kThreads) cp_async16<0>(ci_stage + 4 * vB0 + 16 * i, ciB + i, 1);
             for (int i = t; i < ngtA; i += kThreads) cp_async4(to_stage + 4 * i, p.tileoffset + gA + i);
@@ -395,7 +400,7 @@ spmspv_kernel(const Params p) {
             unsigned base = __reduce_add_sync(0xFFFFFFFFu, lane < warp ? tl : 0u);          // before my first group
             nact = static_cast<int>(total);
             nactA_pad = (ngtB > 0) ? static_cast<int>(realA + pad) : ((nact + kGroup - 1) / kGroup) * kGroup;
-            const int64_t slotA0 = gA * kTileK - jA0, slotB0 = gB * kTileK;                  // column slot of column 0
+            const unsigned slotA0 = gA * kTileK - jA0, slotB0 = gB * kTileK;                 // column slot of column 0
 #pragma unroll
             for (int k = 0; k < kMaxGroupsPerWarp; ++k) {
                 const int q = warp * gpw + k;
@@ -403,7 +408,7 @@ spmspv_kernel(const Params p) {
                 if ((m >> lane) & 1u) {
                     const int v = q * 32 + lane;
                     const int j = (v < vB0) ? jA0 + v : v - vB0;
-                    const unsigned slot = static_cast<unsigned>((v < vB0 ? slotA0 : slotB0) + j);
+                    const unsigned slot = (v < vB0 ? slotA0 : slotB0) + j;
                     const int item = static_cast<int>(base + (q >= qB ? pad : 0u) + __popc(m & ((1u << lane) - 1u)));
                     const uint32_t ci = sm.stage.colinfo[v];                                // ColInfo: offset << 16 | nnz
                     sm.rec[item] = make_uint2(sm.stage.tileoff[v >> 4] + (ci >> 16), (slot << 6) | (((ci & 0xFFFFu) + 7u) >> 3));
@@ -422,22 +427,25 @@ spmspv_kernel(const Params p) {
 
         // ---- (2) per-warp fetch / decode pipeline over groups warp, warp + kWarps, ... ----
         const int groupsA = nactA_pad / kGroup;                 // groups [0, groupsA) belong to piece A
-        // fetch(i): start the copies of my i-th group into ring position i % kDepth
-        auto fetch = [&](int i) {
-            const int lq = warp + i * kWarps;
-            if (lq < ngroups) {
-                const int d = i % kDepth;
-                const uint2 rc = lds_v2(rec_addr + 8u * (lq * kGroup + lgrp));
-                const uint32_t bdst = bm_own + d * 128;
+        // Carried from group to group: lq = the group being decoded, (dv, db) = its ring position as
+        // byte offsets into the values ring / the bitmap table, rec_nxt = my record of the next group to fetch.
+        int lq = warp;
+        uint32_t dv = 0, db = 0;
+        uint32_t rec_nxt = rec_addr + 8u * (warp * kGroup + lgrp);
+        // start the copies of group glq (my record at rec_a) into ring position (dv_f, db_f)
+        auto fetch_group = [&](int glq, uint32_t rec_a, uint32_t dv_f, uint32_t db_f) {
+            if (glq < ngroups) {
+                const uint2 rc = lds_v2(rec_a);
+                const uint32_t bdst = bm_own + db_f;
                 if (rc.y != kNullRec) {
                     const int rem = static_cast<int>(rc.y & 63u) - lane7;                  // my 16-byte pieces left
-                    const unsigned char* src = val_src + 2 * static_cast<uint64_t>(rc.x);
-                    const uint32_t dst = val_dst + d * kStageBytes;
+                    const unsigned char* src = reinterpret_cast<const unsigned char*>(p.values) + (2 * static_cast<uint64_t>(rc.x) + 16u * lane7);
+                    const uint32_t dst = val_dst + dv_f;
                     cp_async16<0>(dst, src, rem);
                     cp_async16<128>(dst, src, rem);
                     cp_async16<256>(dst, src, rem);
                     cp_async16<384>(dst, src, rem);
-                    cp_async4(bdst, bm_src + static_cast<size_t>(rc.y >> 6) * 32);
+                    cp_async4(bdst, reinterpret_cast<const unsigned char*>(p.bitmap) + (static_cast<size_t>(rc.y >> 6) * 32 + 4u * lane7));
                 } else {
                     sts_u32(bdst, 0u);
                 }
@@ -445,53 +453,49 @@ spmspv_kernel(const Params p) {
             cp_async_commit();
         };
 #pragma unroll
-        for (int d = 0; d < kDepth; ++d) fetch(d);
-
-        int d = 0;
-        bool in_first = (ngtB > 0);                             // still inside piece A of a two-piece batch
-        for (int i = 0, lq = warp; lq < ngroups; ++i, lq += kWarps) {
-            if (in_first && lq >= groupsA) {
-                // my share of piece A is complete: park it and start piece B's row tile from zero
-                in_first = false;
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    sm.red_first[warp][4 * lane + k] = acc[k];
-                    sm.red_first[warp][128 + 4 * lane + k] = acc[4 + k];
-                    acc[k] = 0.f;
-                    acc[4 + k] = 0.f;
-                }
-            }
+        for (int dd = 0; dd < kDepth; ++dd) {
+            fetch_group(warp + dd * kWarps, rec_nxt, dd * kStageBytes, dd * 128);
+            rec_nxt += 8u * kGroup * kWarps;
+        }
+        const unsigned m1 = bit0 << 1, m2 = bit0 << 2, m3 = bit0 << 3;
+        // one group: wait for its copies, scan, decode, refill its ring position with the group kDepth ahead
+        auto one_group = [&]() {
             cp_async_wait<kDepth - 1>();
             __syncwarp();
-            // scan role: shared address of my word's first value
-            {
-                const unsigned cnt = __popc(lds_u32(bm_own + d * 128));
+            {   // scan role: offset of my word's first value inside the warp's ring
+                const unsigned cnt = __popc(lds_u32(bm_own + db));
                 unsigned inc = cnt;
-#pragma unroll
-                for (int dd = 1; dd < 8; dd <<= 1) {
-                    unsigned v = __shfl_up_sync(0xFFFFFFFFu, inc, dd, 8);
-                    if (lane7 >= dd) inc += v;
-                }
-                sts_u16(vo_own, lgrp * kSlotBytes + d * kStageBytes + 2u * (inc - cnt));
+                scan8_level<1>(inc);
+                scan8_level<2>(inc);
+                scan8_level<4>(inc);
+                sts_u16(vo_own, slot_off + dv + 2u * (inc - cnt));
             }
             __syncwarp();
-            // decode role: my 8 words (tile it, word 4h + lgrp at index 2*it + h), their value addresses, the 4 x
-            const unsigned m1 = bit0 << 1, m2 = bit0 << 2, m3 = bit0 << 3;
+            // decode role: my 8 words (tile it, word 4h + lgrp at index 2*it + h), their value offsets, the 4 x
+            const uint32_t x_cur = x_addr + 8u * lq;
 #pragma unroll 1
             for (int half = 0; half < 2; ++half) {
-                const uint4 w = lds_v4(bm_dec + d * 128 + 16 * half);
+                const uint4 w = lds_v4(bm_dec + db + 16 * half);
                 const uint2 a = lds_v2(vo_dec + 8 * half);                       // four 16-bit offsets
-                const unsigned xs = lds_u32(x_addr + 8u * lq + 4 * half);        // two activations
+                const unsigned xs = lds_u32(x_cur + 4 * half);                   // two activations
                 decode_step(w.x, ring_w + (a.x & 0xFFFFu), lt_mask, bit0, m1, m2, m3, xs, acc[0], acc[1], acc[2], acc[3]);
                 decode_step(w.y, ring_w + (a.x >> 16), lt_mask, bit0, m1, m2, m3, xs, acc[4], acc[5], acc[6], acc[7]);
                 decode_step(w.z, ring_w + (a.y & 0xFFFFu), lt_mask, bit0, m1, m2, m3, xs >> 16, acc[0], acc[1], acc[2], acc[3]);
                 decode_step(w.w, ring_w + (a.y >> 16), lt_mask, bit0, m1, m2, m3, xs >> 16, acc[4], acc[5], acc[6], acc[7]);
             }
-            __syncwarp();                  // everyone is done with ring position d
-            fetch(i + kDepth);
-            d = (d + 1 == kDepth) ? 0 : d + 1;
-        }
-        if (in_first) {                    // this warp had no group of piece B: its piece-A sums are still in registers
+            __syncwarp();                  // everyone is done with this ring position
+            fetch_group(lq + kDepth * kWarps, rec_nxt, dv, db);
+            rec_nxt += 8u * kGroup * kWarps;
+            lq += kWarps;
+            if (kDepth == 2) {
+                dv ^= kStageBytes;
+                db ^= 128u;
+            } else {
+                dv = (dv == (kDepth - 1) * kStageBytes) ? 0u : dv + kStageBytes;
+                db = (db == (kDepth - 1) * 128u) ? 0u : db + 128u;
+            }
+        };
+        auto park_first = [&]() {      // my share of the first piece is complete: park it, restart from zero
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
                 sm.red_first[warp][4 * lane + k] = acc[k];
@@ -499,7 +503,16 @@ spmspv_kernel(const Params p) {
                 acc[k] = 0.f;
                 acc[4 + k] = 0.f;
             }
+        };
+        bool in_first = (ngtB > 0);
+        while (lq < ngroups) {
+            if (in_first && lq >= groupsA) {
+                in_first = false;
+                park_first();
+            }
+            one_group();
         }
+        if (in_first) park_first();
         cp_async_wait<0>();
         __syncthreads();       // all pipelines drained: the ring is idle
 

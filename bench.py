@@ -63,6 +63,22 @@ def active_bytes(colinfo: np.ndarray, active_words: np.ndarray, M: int, K: int, 
     return int(per_tile[:, act].sum()) + 4 * (gt + 1) + 2 * K + y_bytes * M
 
 
+def max_over_ranks(x: float, world: int, device="cuda") -> float:
+    """The slowest rank's time: a MAX all-reduce over the process group (identity for one rank)."""
+    if world <= 1:
+        return float(x)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def replica_value(bytes_per_step: int, world: int, ms_per_step: float) -> float:
+    """Whole-job effective GB/s of `world` independent replicas that each move bytes_per_step."""
+    return world * bytes_per_step / (ms_per_step * 1e-3) / 1e9
+
+
 def measured_peak():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -253,12 +269,9 @@ def main():
     ms = ev0.elapsed_time(ev1)
     clocks = sampler.stop()
     assert all(spdp.spdp_last_device_status(h) == 0 for h in handles)
-    if world > 1:
-        tmax = torch.tensor([ms], device="cuda")
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        ms = float(tmax.item())
+    ms = max_over_ranks(ms, world)
     ms_per_step = ms / args.steps
-    value = world * B_active / (ms_per_step * 1e-3) / 1e9
+    value = replica_value(B_active, world, ms_per_step)
 
     # ---- end to end through the host-vector entry point ----------------------------------
     xh = torch.from_numpy(w.x.copy()).pin_memory()
@@ -272,11 +285,8 @@ def main():
         spdp.spdp_spmspv_host(handles[i % copies], xh, w.rule, w.thr, yh)
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
-    if world > 1:
-        tmax = torch.tensor([e2e_s], device="cuda", dtype=torch.float64)
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        e2e_s = float(tmax.item())
-    e2e_value = world * B_active * e2e_steps / e2e_s / 1e9
+    e2e_s = max_over_ranks(e2e_s, world)
+    e2e_value = replica_value(B_active, world, e2e_s / e2e_steps * 1e3)
 
     if rank != 0:
         if world > 1:

@@ -79,6 +79,8 @@ spdp_status build_partition(spdp_matrix* h, int num_ctas) {
 spdp_status finish_handle(spdp_matrix* h) {
     spdp_status st = build_partition(h, 0);
     if (st != SPDP_OK) return st;
+    st = configure_spmspv_kernel();
+    if (st != SPDP_OK) return st;
     SPDP_CUDA_TRY(cudaMalloc(&h->status_word, sizeof(int)));
     SPDP_CUDA_TRY(cudaMemset(h->status_word, 0, sizeof(int)));
     SPDP_CUDA_TRY(cudaMalloc(&h->x_stage, h->K * sizeof(__half)));
@@ -179,6 +181,8 @@ spdp_status spdp_spmspv(spdp_handle h, const void* x_dev, spdp_dp_rule rule, flo
         (reinterpret_cast<uintptr_t>(mask_dev) & 3u))
         return SPDP_ERR_INVALID_ARG;
     if (h->pad_elems != 8) return SPDP_ERR_UNSUPPORTED_SHAPE;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev != h->device) return SPDP_ERR_INVALID_ARG;   // wrong current device
     return launch_spmspv(h, static_cast<const __half*>(x_dev), rule, thr,
                          static_cast<const uint32_t*>(mask_dev), y_dev, ydt, static_cast<cudaStream_t>(stream));
 }

@@ -68,6 +68,7 @@ spdp_status unpack_device(const spdp_matrix* h, __half* W, int64_t ldw, cudaStre
 
 // spmspv.cu
 int default_ctas_per_sm();   // CTAs of the spMspV kernel that share one SM
+spdp_status configure_spmspv_kernel();   // per-device kernel attributes; idempotent
 spdp_status launch_spmspv(const spdp_matrix* h, const __half* x, int rule, float thr,
                           const uint32_t* mask, void* y, int ydt, cudaStream_t s);
 spdp_status launch_spmspv_noalloc(const uint32_t* tileoffset, const uint32_t* colinfo, const uint64_t* bitmap,

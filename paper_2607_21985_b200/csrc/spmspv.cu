@@ -540,19 +540,11 @@ spmspv_kernel(const Params p) {
     }
 }
 
-// Launch helper shared by the entry points: opts in to the large dynamic shared memory once per
-// device, then launches P CTAs.
+// Launch helper shared by the entry points.
 spdp_status launch_kernel(const Params& p, int num_ctas, cudaStream_t s) {
-    constexpr size_t kSmemBytes = sizeof(Smem);
-    static bool configured[64] = {};
-    int dev = 0;
-    SPDP_CUDA_TRY(cudaGetDevice(&dev));
-    if (dev < 0 || dev >= 64 || !configured[dev]) {
-        SPDP_CUDA_TRY(cudaFuncSetAttribute(spmspv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           static_cast<int>(kSmemBytes)));
-        if (dev >= 0 && dev < 64) configured[dev] = true;
-    }
-    spmspv_kernel<<<num_ctas, kThreads, kSmemBytes, s>>>(p);
+    spdp_status st = configure_spmspv_kernel();        // a flag test after the first call on a device
+    if (st != SPDP_OK) return st;
+    spmspv_kernel<<<num_ctas, kThreads, sizeof(Smem), s>>>(p);
     SPDP_CUDA_TRY(cudaGetLastError());
     return SPDP_OK;
 }
@@ -595,6 +587,23 @@ __global__ void noalloc_setup_kernel(NoAllocScratch* sc, int R) {
 }  // namespace
 
 int default_ctas_per_sm() { return kCtasPerSm; }
+
+// Opts the kernel in to its large dynamic shared memory, once per device (handle creation calls
+// this, so spdp_spmspv itself only launches).
+spdp_status configure_spmspv_kernel() {
+    static std::mutex mu;
+    static bool configured[64] = {};
+    int dev = 0;
+    SPDP_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return SPDP_ERR_UNSUPPORTED_SHAPE;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!configured[dev]) {
+        SPDP_CUDA_TRY(cudaFuncSetAttribute(spmspv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           static_cast<int>(sizeof(Smem))));
+        configured[dev] = true;
+    }
+    return SPDP_OK;
+}
 
 spdp_status launch_spmspv(const spdp_matrix* h, const __half* x, int rule, float thr,
                           const uint32_t* mask, void* y, int ydt, cudaStream_t s) {

@@ -239,6 +239,53 @@ def test_spmspv_degenerate_cases(S):
         S.spdp_free(h)
 
 
+def test_unaligned_x_and_mask_rule_on_a_long_row(S):
+    """x that is only 2-byte aligned takes the kernel's plain-load path; the explicit mask rule on two batches."""
+    w = WL.config2(768, 9000, seed=8)
+    a = O.active_ref(w.x, w.rule, w.thr)
+    y_ref, S_ref = O.spmspv_ref(w.W, w.x, a)
+    h = S.spdp_pack_tiled_cbc(dev(w.W))
+    try:
+        buf = torch.zeros(w.K + 8, dtype=torch.float16, device="cuda")
+        for shift in (1, 3, 8):
+            xs = buf[shift: shift + w.K]
+            xs.copy_(dev(w.x))
+            assert xs.data_ptr() % 16 == (2 * shift) % 16
+            y = torch.full((w.M,), float("nan"), dtype=torch.float32, device="cuda")
+            S.spdp_spmspv(h, xs, w.rule, w.thr, y)
+            torch.cuda.synchronize()
+            check_y(y.cpu().numpy().astype(np.float64), y_ref, S_ref)
+        y = gpu_spmspv(S, h, w.x, O.DP_MASK, 0.0, w.M, mask_words=O.active_to_words(a))
+        check_y(y, y_ref, S_ref)
+    finally:
+        S.spdp_free(h)
+
+
+def test_spmspv_in_a_cuda_graph(S):
+    """spdp_spmspv only launches (no allocation, no synchronisation): it can be captured and replayed."""
+    w = WL.config1(1024, 2048, seed=9)
+    a = O.active_ref(w.x, w.rule, w.thr)
+    y_ref, S_ref = O.spmspv_ref(w.W, w.x, a)
+    h = S.spdp_pack_tiled_cbc(dev(w.W))
+    try:
+        x = dev(w.x)
+        y = torch.zeros(w.M, dtype=torch.float32, device="cuda")
+        S.spdp_spmspv(h, x, w.rule, w.thr, y)                      # warm-up outside the capture
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        side = torch.cuda.Stream()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g, stream=side):
+                S.spdp_spmspv(h, x, w.rule, w.thr, y, stream=side)
+        for _ in range(3):
+            y.fill_(float("nan"))
+            g.replay()
+            torch.cuda.synchronize()
+            check_y(y.cpu().numpy().astype(np.float64), y_ref, S_ref)
+    finally:
+        S.spdp_free(h)
+
+
 def test_imported_oracle_arrays_give_same_result(S):
     w = WL.config1(768, 640, seed=4)
     p = O.pack_fast(w.W)

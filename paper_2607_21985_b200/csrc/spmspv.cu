@@ -78,8 +78,10 @@ struct __align__(128) Smem {
     };
     // Bitmap words of a group in decode order: word w of the group's it-th tile sits at
     // [(w & 3) * 8 + it * 2 + (w >> 2)], so the lanes that decode words (w & 3) == g read 8 consecutive words.
-    alignas(16) uint32_t bmring[kWarps][kDepth][32];
-    alignas(16) unsigned short voff[kWarps][32];        // same order: byte offset of each word's first value in the warp's ring
+    struct alignas(16) WarpTab {
+        uint32_t bm[kDepth][32];
+        unsigned short voff[32];                        // same order: byte offset of each word's first value in the warp's ring
+    } tab[kWarps];
     // Active list of the chunk, one record per active column tile (filled once per chunk):
     alignas(16) uint2 rec[kChunkCols + kGroup];         // .x = start of its values in Values (elements),
                                                         // .y = (column slot in Bitmap/ColInfo) << 6 | 16-byte pieces
@@ -89,8 +91,7 @@ struct __align__(128) Smem {
     uint32_t warp_total[kWarps][2];                     // list phase: records listed by each warp (all, piece A)
     int is_last[2];
 };
-static_assert(offsetof(Smem, rec) % 16 == 0 && offsetof(Smem, xact) % 16 == 0 && offsetof(Smem, voff) % 16 == 0 &&
-              offsetof(Smem, bmring) % 16 == 0, "16-byte shared loads need aligned tables");
+static_assert(offsetof(Smem, rec) % 16 == 0 && offsetof(Smem, xact) % 16 == 0 && offsetof(Smem, tab) % 16 == 0, "16-byte shared loads need aligned tables");
 static_assert(sizeof(float) * kWarps * kTileM <= size_t(kWarps) * kDepth * kStageBytes, "red must fit in the ring");
 static_assert(sizeof(uint32_t) * (kChunkCols + kChunkGT) + 2 * kChunkCols + sizeof(float) * kWarps * kTileM <=
                   size_t(kWarps) * kDepth * kStageBytes,
@@ -110,6 +111,13 @@ __device__ __forceinline__ void store_y(void* y, int ydt, int64_t i, float v) {
     else static_cast<__half*>(y)[i] = __float2half_rn(v);
 }
 
+// Makes a loop-invariant value opaque to the compiler, so that it stays in its register instead of
+// being recomputed from the thread index inside the hot loop.
+template <typename T>
+__device__ __forceinline__ T pinned(T v) {
+    asm volatile("" : "+r"(v));
+    return v;
+}
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
@@ -282,19 +290,21 @@ spmspv_kernel(const Params p) {
 
     const int lane7 = lane & 7;
     const int lgrp = lane >> 3;
-    const unsigned bit0 = 1u << (4 * lane7);        // first bit of my nibble inside a 32-bit bitmap word
-    const unsigned lt_mask = bit0 - 1u;
+    const unsigned bit0 = pinned(1u << (4 * lane7));    // first bit of my nibble inside a 32-bit bitmap word
+    const unsigned lt_mask = pinned(bit0 - 1u);
     // fetch role: lane (lgrp, lane7) moves 16-byte pieces lane7, lane7+8, ... and bitmap word lane7 of the
     // group's lgrp-th tile.  scan role: the same (tile, word).  decode role: nibble lane7 of words w with
     // (w & 3) == lgrp of every tile of the group.
     const int tpos = (lane7 & 3) * 8 + lgrp * 2 + (lane7 >> 2);         // where (tile lgrp, word lane7) sits
-    const uint32_t val_dst = smem_u32(&sm.ring[warp][0][lgrp * kSlotBytes + 16 * lane7]);
-    const uint32_t bm_own = smem_u32(&sm.bmring[warp][0][tpos]);
-    const uint32_t bm_dec = smem_u32(&sm.bmring[warp][0][lgrp * 8]);
-    const uint32_t vo_own = smem_u32(&sm.voff[warp][tpos]);
-    const uint32_t vo_dec = smem_u32(&sm.voff[warp][lgrp * 8]);
-    const uint32_t ring_w = smem_u32(&sm.ring[warp][0][0]);                         // my warp's ring
-    const uint32_t slot_off = lgrp * kSlotBytes;                                    // scan role: my tile's slot in a stage
+    const uint32_t val_dst = pinned(smem_u32(&sm.ring[warp][0][lgrp * kSlotBytes + 16 * lane7]));
+    const uint32_t bm_own = pinned(smem_u32(&sm.tab[warp].bm[0][tpos]));
+    const uint32_t bm_dec = pinned(smem_u32(&sm.tab[warp].bm[0][lgrp * 8]));
+    // voff[i] sits kVoffFromBm - 2*i bytes behind bm[0][i]
+    constexpr uint32_t kVoffFromBm = kDepth * 128;
+    const uint32_t vo_own = bm_own + kVoffFromBm - 2u * tpos;
+    const uint32_t vo_dec = bm_dec + kVoffFromBm - 16u * lgrp;
+    const uint32_t ring_w = pinned(smem_u32(&sm.ring[warp][0][0]));                 // my warp's ring
+    const uint32_t slot_off = pinned(static_cast<uint32_t>(lgrp * kSlotBytes));     // scan role: my tile's slot in a stage
     const uint32_t rec_addr = smem_u32(&sm.rec[0]);
     const uint32_t x_addr = smem_u32(&sm.xact[0]);
 
@@ -457,7 +467,7 @@ spmspv_kernel(const Params p) {
             fetch_group(warp + dd * kWarps, rec_nxt, dd * kStageBytes, dd * 128);
             rec_nxt += 8u * kGroup * kWarps;
         }
-        const unsigned m1 = bit0 << 1, m2 = bit0 << 2, m3 = bit0 << 3;
+        const unsigned m1 = pinned(bit0 << 1), m2 = pinned(bit0 << 2), m3 = pinned(bit0 << 3);
         // one group: wait for its copies, scan, decode, refill its ring position with the group kDepth ahead
         auto one_group = [&]() {
             cp_async_wait<kDepth - 1>();

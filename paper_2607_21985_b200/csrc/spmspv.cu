@@ -308,6 +308,10 @@ spmspv_kernel(const Params p) {
     const uint32_t rec_addr = smem_u32(&sm.rec[0]);
     const uint32_t x_addr = smem_u32(&sm.xact[0]);
 
+    // Let a dependent launch (the next call) begin as soon as SMs free up.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    bool waited_for_stream = false;  // x, y, workspace and counters may belong to the previous kernel until we wait
+
     float acc[8];                   // rows 4*lane+k (k<4) and 128+4*lane+(k-4) of the current row tile
 #pragma unroll
     for (int k = 0; k < 8; ++k) acc[k] = 0.f;
@@ -355,6 +359,11 @@ spmspv_kernel(const Params p) {
             for (int i = t; i < ngtB * (kTileK / 4); i += kThreads) cp_async16<0>(ci_stage + 4 * vB0 + 16 * i, ciB + i, 1);
             for (int i = t; i < ngtA; i += kThreads) cp_async4(to_stage + 4 * i, p.tileoffset + gA + i);
             for (int i = t; i < ngtB; i += kThreads) cp_async4(to_stage + (vB0 >> 2) + 4 * i, p.tileoffset + gB + i);
+            if (!waited_for_stream) {
+                // everything above reads only the packed matrix; from here on the previous kernel's results count
+                asm volatile("griddepcontrol.wait;" ::: "memory");
+                waited_for_stream = true;
+            }
             if ((reinterpret_cast<uintptr_t>(p.x) & 15u) == 0) {
                 // list position v holds x[jA0 + v] (piece A) or x[v - vB0] (piece B); 8 activations per copy
                 for (int i = t; 8 * i < nA; i += kThreads)
@@ -550,12 +559,25 @@ spmspv_kernel(const Params p) {
     }
 }
 
-// Launch helper shared by the entry points.
+// Launch helper shared by the entry points.  The launch carries the programmatic-stream-serialization
+// attribute: the CTAs of this kernel may start while the previous kernel in the stream is still
+// draining, stage the matrix metadata of their range (which no kernel in the stream writes), and
+// only then wait for the previous kernel (griddepcontrol.wait) before they touch x, y or the
+// workspace.  Back-to-back calls overlap one call's tail with the next call's prologue.
 spdp_status launch_kernel(const Params& p, int num_ctas, cudaStream_t s) {
     spdp_status st = configure_spmspv_kernel();        // a flag test after the first call on a device
     if (st != SPDP_OK) return st;
-    spmspv_kernel<<<num_ctas, kThreads, sizeof(Smem), s>>>(p);
-    SPDP_CUDA_TRY(cudaGetLastError());
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(num_ctas));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = sizeof(Smem);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    SPDP_CUDA_TRY(cudaLaunchKernelEx(&cfg, spmspv_kernel, p));
     return SPDP_OK;
 }
 

@@ -136,13 +136,13 @@ SPDP_API spdp_status spdp_spmspv_host(spdp_handle h, const void* x_host, spdp_dp
  * handle; the caller passes the packed arrays (device pointers, laid out as spdp_info describes,
  * 16-byte column padding), x, the DP rule and y, exactly as for spdp_spmspv.
  *
- * What spdp_spmspv keeps in handle-owned allocations (CTA ranges, per-row-tile tables, arrival
- * counters, split-K partial sums) lives in ONE fixed device array inside the library, about
- * 1.1 MB, present on every GPU that loads the library until the process exits.  Limits: at most
- * 4096 row tiles (M <= 1,048,576); larger shapes return SPDP_ERR_UNSUPPORTED_SHAPE.  At most 512
- * CTAs are launched.  The call enqueues a small set-up kernel (which also clears the counters the
- * previous call left behind) and the spMspV kernel on `stream`; it calls no cudaMalloc, cudaFree or
- * allocating library routine.
+ * What spdp_spmspv keeps in a handle-owned allocation (the split-K partial sums that CTAs
+ * exchange) lives in ONE fixed device array inside the library, about 0.5 MB, present on every
+ * GPU that loads the library until the process exits.  It bounds the launch to 512 CTAs (the
+ * library never asks for more); shapes beyond the library's general limit (2^26 column tiles)
+ * return SPDP_ERR_UNSUPPORTED_SHAPE.  The call enqueues a small set-up kernel (which empties the
+ * part of the array this call uses, whatever an earlier call left there) and the spMspV kernel
+ * on `stream`; it calls no cudaMalloc, cudaFree or allocating library routine.
  *
  * The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
  * that device current) and the SM count; make that first call outside any stream capture.

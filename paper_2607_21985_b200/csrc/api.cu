@@ -26,7 +26,6 @@ void release(spdp_matrix* h) {
     cudaFree(h->bitmap);
     cudaFree(h->values);
     cudaFree(h->workspace);
-    cudaFree(h->row_counter);
     cudaFree(h->status_word);
     cudaFree(h->x_stage);
     cudaFree(h->mask_stage);
@@ -58,21 +57,18 @@ spdp_status new_handle(int64_t M, int64_t K, int pad_elems, spdp_matrix** out) {
 }
 
 // Chooses the number of CTAs (the kernel cuts the NGT GTiles into that many equal contiguous
-// ranges) and (re)allocates what depends on it: the split-K workspace and the arrival counters.
+// ranges) and (re)allocates what depends on it: the split-K workspace (all zero = every tree node empty).
 spdp_status build_partition(spdp_matrix* h, int num_ctas) {
-    const int64_t NGT = h->NGT, R = h->R;
+    const int64_t NGT = h->NGT;
     int P = num_ctas > 0 ? num_ctas : h->sm_count * default_ctas_per_sm();
     if (P > 1024) P = 1024;          // the kernel's range arithmetic is 32-bit: NGT < 2^22 times P must fit
     if (P > NGT) P = static_cast<int>(NGT);
     if (P < 1) P = 1;
     cudaFree(h->workspace);     h->workspace = nullptr;
-    cudaFree(h->row_counter);   h->row_counter = nullptr;
     h->num_ctas = P;
-    h->workspace_bytes = static_cast<int64_t>(P) * 2 * kTileM * sizeof(float);   // two slots per CTA
+    h->workspace_bytes = static_cast<int64_t>(P) * kTileM * sizeof(float);   // one row of split-K tree nodes per CTA
     SPDP_CUDA_TRY(cudaMalloc(&h->workspace, h->workspace_bytes));
-    SPDP_CUDA_TRY(cudaMalloc(&h->row_counter, R * sizeof(unsigned)));
     SPDP_CUDA_TRY(cudaMemset(h->workspace, 0, h->workspace_bytes));
-    SPDP_CUDA_TRY(cudaMemset(h->row_counter, 0, R * sizeof(unsigned)));
     return SPDP_OK;
 }
 

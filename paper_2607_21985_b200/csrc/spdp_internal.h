@@ -35,8 +35,7 @@ struct spdp_matrix {
     // Work partition of one spmspv launch: the kernel cuts the NGT GTiles into num_ctas equal
     // contiguous ranges, one per CTA.
     int num_ctas;           // P
-    float* workspace;       // device [P*2*256] split-K partial sums (two slots per CTA)
-    unsigned* row_counter;  // device [R] arrivals per row tile (self-resetting)
+    float* workspace;       // device [P*256] split-K tree nodes, one row per CTA (all zero between calls)
     int* status_word;       // device [1]
     int64_t workspace_bytes;
 

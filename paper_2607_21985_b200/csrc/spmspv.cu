@@ -5,11 +5,11 @@
 // row-major storage order, are cut into num_ctas equal contiguous ranges, one per CTA.  A range
 // touches one or more row tiles; each (CTA, row tile) piece is a "segment" that yields 256
 // fp32 partial sums.  A row tile fed by one segment is written to y directly; otherwise the
-// partials go to the handle's workspace (the paper's ReductionWorkspace) and the CTA that
-// arrives last at the row tile's counter adds them in segment order -- no CTA ever waits for
-// another, and the order of the additions is fixed.  Only the first and the last segment of a
-// CTA can share their row tile with another CTA, so a CTA owns two workspace slots: slot 0 for
-// the row tile its range starts in, slot 1 for any later one.
+// segments' partials are added pairwise along a fixed binary tree through the handle's
+// workspace (the paper's ReductionWorkspace): whoever reaches a tree node first leaves its sum
+// there with one atomic exchange, the second takes it, adds, and moves up; the thread that
+// completes the root stores y.  No CTA ever waits for another, and the shape of the tree, hence
+// the rounding of the result, does not depend on who arrives when.
 #include <cstddef>
 #include <mutex>
 
@@ -33,6 +33,12 @@ namespace {
 #ifndef SPDP_DEPTH
 #define SPDP_DEPTH 2
 #endif
+#ifndef SPDP_PIN_SRC
+#define SPDP_PIN_SRC 3
+#endif
+#ifndef SPDP_UNROLL_HALF
+#define SPDP_UNROLL_HALF 0
+#endif
 constexpr int kWarps = SPDP_WARPS;         // warps per CTA; every warp fetches and decodes its own column tiles
 constexpr int kDepth = SPDP_DEPTH;         // groups a warp keeps in flight
 constexpr int kGroup = 4;                  // active column tiles per group (one fetch / decode unit of a warp)
@@ -45,6 +51,7 @@ constexpr int kCtasPerSm = SPDP_CTAS_PER_SM;
 constexpr uint32_t kNullRec = 0xFFFFFFFFu;
 constexpr int kMaxGroupsPerWarp = (kChunkCols / 32 + kWarps - 1) / kWarps;   // 32-position groups a warp lists per batch
 constexpr int kChunkGT = kChunkCols / kTileK;
+constexpr int kRecPad = kGroup * (kDepth * kWarps + 1);   // null records behind the last real one
 
 struct Params {
     const uint32_t* tileoffset;
@@ -60,8 +67,7 @@ struct Params {
     int M, K, R, C;
     int64_t NGT;            // R * C GTiles, cut into num_ctas equal contiguous ranges
     int num_ctas;
-    float* workspace;
-    unsigned* row_counter;
+    float* workspace;       // [num_ctas][256] tree nodes of the split-K combine, all zero between calls
     int* status;
 };
 
@@ -77,19 +83,20 @@ struct __align__(128) Smem {
         } stage;
     };
     // Bitmap words of a group in decode order: word w of the group's it-th tile sits at
-    // [(w & 3) * 8 + it * 2 + (w >> 2)], so the lanes that decode words (w & 3) == g read 8 consecutive words.
+    // [(w & 1) * 16 + it * 4 + (w >> 1)], so the lanes that decode the even (odd) words read 16 consecutive words.
     struct alignas(16) WarpTab {
         uint32_t bm[kDepth][32];
-        unsigned short voff[32];                        // same order: byte offset of each word's first value in the warp's ring
+        uint32_t vo[kDepth][32];                        // same order: shared-memory address of each word's first value
     } tab[kWarps];
     // Active list of the chunk, one record per active column tile (filled once per chunk):
-    alignas(16) uint2 rec[kChunkCols + kGroup];         // .x = start of its values in Values (elements),
+    alignas(16) uint2 rec[kChunkCols + kRecPad];        // .x = start of its values in Values (elements),
                                                         // .y = (column slot in Bitmap/ColInfo) << 6 | 16-byte pieces
-                                                        //      of values; kNullRec pads a piece to whole groups
+                                                        //      of values; kNullRec pads a piece to whole groups and
+                                                        //      follows the last record for kRecPad entries, so a warp
+                                                        //      can fetch kDepth groups ahead without a range test
     alignas(16) unsigned short xact[kChunkCols + kGroup];   // its activation x_j (fp16 bits)
     float red_first[kWarps][kTileM];                    // row reduction of a batch's first piece (flushed mid-stream)
     uint32_t warp_total[kWarps][2];                     // list phase: records listed by each warp (all, piece A)
-    int is_last[2];
 };
 static_assert(offsetof(Smem, rec) % 16 == 0 && offsetof(Smem, xact) % 16 == 0 && offsetof(Smem, tab) % 16 == 0, "16-byte shared loads need aligned tables");
 static_assert(sizeof(float) * kWarps * kTileM <= size_t(kWarps) * kDepth * kStageBytes, "red must fit in the ring");
@@ -97,6 +104,7 @@ static_assert(sizeof(uint32_t) * (kChunkCols + kChunkGT) + 2 * kChunkCols + size
                   size_t(kWarps) * kDepth * kStageBytes,
               "staging must fit in the ring behind red");
 static_assert(sizeof(Smem) <= (227 * 1024) / kCtasPerSm - 1024 * (kCtasPerSm - 1), "shared memory of one CTA");
+static_assert(kRecPad <= kThreads, "one thread per trailing null record");
 static_assert(kWarps >= 16, "two groups of 256 threads finish two row tiles side by side");
 
 // DP test of Sec. 4.2 step (3): magnitude against the threshold; NOT(|x| <= thr) keeps NaN.
@@ -115,7 +123,8 @@ __device__ __forceinline__ void store_y(void* y, int ydt, int64_t i, float v) {
 // being recomputed from the thread index inside the hot loop.
 template <typename T>
 __device__ __forceinline__ T pinned(T v) {
-    asm volatile("" : "+r"(v));
+    if constexpr (sizeof(T) == 8) asm volatile("" : "+l"(v));
+    else asm volatile("" : "+r"(v));
     return v;
 }
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -138,49 +147,48 @@ __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commi
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-// One decode step (Sec. 4.2.1): the 4 consecutive rows this lane owns inside the 32-bit bitmap
+// One decode step (Sec. 4.2.1): the 2 consecutive rows this lane owns inside the 32-bit bitmap
 // word W.  `first` is the shared-memory address of the word's first value, `below` masks the bits
-// of lower nibbles, m0..m3 are the lane's four bits.  rank = set bits before the position; a set
+// of lower rows, m0 and m1 are the lane's two bits.  rank = set bits before the position; a set
 // bit takes the next value and adds value * x to its row's fp32 accumulator.  fma.rn.f32.f16
-// multiplies two fp16 exactly and accumulates in fp32.
-__device__ __forceinline__ void decode_step(unsigned W, uint32_t first, unsigned below, unsigned m0, unsigned m1,
-                                            unsigned m2, unsigned m3, unsigned x32, float& a0, float& a1,
-                                            float& a2, float& a3) {
-    asm volatile(
-        "{\n"
-        " .reg .pred p0, p1, p2, p3;\n"
-        " .reg .b16 v0, v1, v2, v3, xl, xu;\n"
-        " .reg .b32 t, a;\n"
-        " and.b32 t, %4, %6;\n"
-        " popc.b32 t, t;\n"
-        " shl.b32 t, t, 1;\n"
-        " add.u32 a, %5, t;\n"
-        " lop3.or.b32 t|p0, %4, %7, 0, 0xC0, 0;\n"
-        " lop3.or.b32 t|p1, %4, %8, 0, 0xC0, 0;\n"
-        " lop3.or.b32 t|p2, %4, %9, 0, 0xC0, 0;\n"
-        " lop3.or.b32 t|p3, %4, %10, 0, 0xC0, 0;\n"
-        " mov.b32 {xl, xu}, %11;\n"
-        " @p0 ld.shared.u16 v0, [a];\n @p0 add.u32 a, a, 2;\n"
-        " @p1 ld.shared.u16 v1, [a];\n @p1 add.u32 a, a, 2;\n"
-        " @p2 ld.shared.u16 v2, [a];\n @p2 add.u32 a, a, 2;\n"
-        " @p3 ld.shared.u16 v3, [a];\n"
+// multiplies two fp16 exactly and accumulates in fp32.  x32 holds two activations; kUpper picks one.
 #if SPDP_FMA_MODE == 0
-        " @p0 fma.rn.f32.f16 %0, v0, xl, %0;\n"
-        " @p1 fma.rn.f32.f16 %1, v1, xl, %1;\n"
-        " @p2 fma.rn.f32.f16 %2, v2, xl, %2;\n"
-        " @p3 fma.rn.f32.f16 %3, v3, xl, %3;\n"
+#define SPDP_FMA2(X)                                  \
+    " @p0 fma.rn.f32.f16 %0, v0, " X ", %0;\n"        \
+    " @p1 fma.rn.f32.f16 %1, v1, " X ", %1;\n"
 #else
-        " .reg .f32 f0, f1, f2, f3, fx;\n"
-        " cvt.f32.f16 fx, xl;\n"
-        " @p0 cvt.f32.f16 f0, v0;\n @p1 cvt.f32.f16 f1, v1;\n @p2 cvt.f32.f16 f2, v2;\n @p3 cvt.f32.f16 f3, v3;\n"
-        " @p0 fma.rn.f32 %0, f0, fx, %0;\n"
-        " @p1 fma.rn.f32 %1, f1, fx, %1;\n"
-        " @p2 fma.rn.f32 %2, f2, fx, %2;\n"
-        " @p3 fma.rn.f32 %3, f3, fx, %3;\n"
+#define SPDP_FMA2(X)                                  \
+    " .reg .f32 f0, f1, fx;\n"                        \
+    " cvt.f32.f16 fx, " X ";\n"                       \
+    " @p0 cvt.f32.f16 f0, v0;\n @p1 cvt.f32.f16 f1, v1;\n" \
+    " @p0 fma.rn.f32 %0, f0, fx, %0;\n"               \
+    " @p1 fma.rn.f32 %1, f1, fx, %1;\n"
 #endif
-        "}"
-        : "+f"(a0), "+f"(a1), "+f"(a2), "+f"(a3)
-        : "r"(W), "r"(first), "r"(below), "r"(m0), "r"(m1), "r"(m2), "r"(m3), "r"(x32));
+#define SPDP_DECODE_BODY(X)                           \
+    "{\n"                                             \
+    " .reg .pred p0, p1;\n"                           \
+    " .reg .b16 v0, v1, xl, xu;\n"                    \
+    " .reg .b32 t, a;\n"                              \
+    " and.b32 t, %2, %4;\n"                           \
+    " popc.b32 t, t;\n"                               \
+    " shl.b32 t, t, 1;\n"                             \
+    " add.u32 a, %3, t;\n"                            \
+    " lop3.or.b32 t|p0, %2, %5, 0, 0xC0, 0;\n"        \
+    " lop3.or.b32 t|p1, %2, %6, 0, 0xC0, 0;\n"        \
+    " mov.b32 {xl, xu}, %7;\n"                        \
+    " @p0 ld.shared.u16 v0, [a];\n @p0 add.u32 a, a, 2;\n" \
+    " @p1 ld.shared.u16 v1, [a];\n"                   \
+    SPDP_FMA2(X)                                      \
+    "}"
+template <bool kUpper>
+__device__ __forceinline__ void decode_step(unsigned W, uint32_t first, unsigned below, unsigned m0, unsigned m1,
+                                            unsigned x32, float& a0, float& a1) {
+    if (kUpper)
+        asm volatile(SPDP_DECODE_BODY("xu")
+                     : "+f"(a0), "+f"(a1) : "r"(W), "r"(first), "r"(below), "r"(m0), "r"(m1), "r"(x32));
+    else
+        asm volatile(SPDP_DECODE_BODY("xl")
+                     : "+f"(a0), "+f"(a1) : "r"(W), "r"(first), "r"(below), "r"(m0), "r"(m1), "r"(x32));
 }
 // One level of an inclusive prefix sum over segments of 8 lanes.
 template <int kDelta>
@@ -193,9 +201,11 @@ __device__ __forceinline__ unsigned lds_u32(uint32_t addr) {
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
     return v;
 }
+template <int kOff>
 __device__ __forceinline__ uint4 lds_v4(uint32_t addr) {
     uint4 v;
-    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4+%5];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr), "n"(kOff));
     return v;
 }
 __device__ __forceinline__ uint2 lds_v2(uint32_t addr) {
@@ -203,11 +213,16 @@ __device__ __forceinline__ uint2 lds_v2(uint32_t addr) {
     asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
     return v;
 }
-__device__ __forceinline__ void sts_u16(uint32_t addr, unsigned v) {
-    asm volatile("{\n .reg .b16 h;\n cvt.u16.u32 h, %1;\n st.shared.u16 [%0], h;\n}" ::"r"(addr), "r"(v) : "memory");
-}
+template <int kOff = 0>
 __device__ __forceinline__ void sts_u32(uint32_t addr, unsigned v) {
-    asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+    asm volatile("st.shared.u32 [%0+%2], %1;" ::"r"(addr), "r"(v), "n"(kOff) : "memory");
+}
+// base + a * kScale with a 64-bit result (one multiply-add)
+template <int kScale>
+__device__ __forceinline__ const unsigned char* offset_wide(const unsigned char* base, uint32_t a) {
+    const unsigned char* r;
+    asm("mad.wide.u32 %0, %1, %2, %3;" : "=l"(r) : "r"(a), "n"(kScale), "l"(base));
+    return r;
 }
 
 // The work split: CTA c owns GTiles [range_begin(c), range_begin(c + 1)) of the row-major GTile order.
@@ -221,46 +236,38 @@ __device__ __forceinline__ int range_owner(const Params& p, unsigned g) {
     return static_cast<int>(((g + 1u) * static_cast<unsigned>(p.num_ctas) + ngt - 1u) / ngt) - 1;
 }
 
-// Adds the kWarps per-warp partial sums of one row tile in warp order and finishes the row tile
-// (256 threads, tt = row inside the tile, `bar` = a named barrier of these 256 threads).  A row tile
-// fed by one segment is stored directly; otherwise the sum goes to this CTA's workspace slot and
-// the CTA that arrives last at the row tile's counter adds all partials in CTA order.
-__device__ __forceinline__ void finish_row_tile(const Params& p, int r, int r_first, const float (*red)[kTileM],
-                                                int tt, int bar, int* is_last) {
+// A partial sum is kept in the workspace XOR this key, so that the all-zero word means "empty".
+// NaN sums are made canonical first, which keeps a stored word from ever being zero.
+constexpr unsigned kNodeKey = 0xFFC0DEADu;
+__device__ __forceinline__ unsigned canonical_bits(float v) { return (v != v) ? 0x7FFFFFFFu : __float_as_uint(v); }
+
+// Adds the kWarps per-warp partial sums of one row tile in warp order and finishes the row (tt =
+// row inside the tile; the rows are independent, nothing here synchronises threads).  A row tile
+// fed by one segment is stored directly.  Otherwise segment i of the row tile's nseg segments is
+// leaf i of a binary tree: at level l, node idx stands for segments [idx << l, (idx + 1) << l); a
+// node without a right-hand neighbour moves up unchanged.  The meeting place of nodes (idx, idx | 1)
+// is the workspace row of the CTA that owns the right node's first segment -- a CTA that starts
+// inside this row tile, and a different one for every tree node.
+__device__ __forceinline__ void finish_row_tile(const Params& p, int r, const float (*red)[kTileM], int tt) {
     float part = 0.f;
 #pragma unroll
     for (int w = 0; w < kWarps; ++w) part += red[w][tt];
     const int64_t row = static_cast<int64_t>(r) * kTileM + tt;
+    if (row >= p.M) return;
     const int q0 = range_owner(p, static_cast<unsigned>(r) * p.C);                 // first and last CTA feeding row tile r
     const int nseg = range_owner(p, static_cast<unsigned>(r + 1) * p.C - 1u) - q0 + 1;
-    if (nseg == 1) {
-        if (row < p.M) store_y(p.y, p.ydt, row, part);
-        return;
+    int idx = static_cast<int>(blockIdx.x) - q0;
+    for (int n = nseg, level = 0; n > 1; n = (n + 1) >> 1, ++level, idx >>= 1) {
+        const int right = idx | 1;
+        if (right >= n) continue;                       // no neighbour at this level
+        unsigned* node = reinterpret_cast<unsigned*>(p.workspace) +
+                         static_cast<int64_t>(q0 + (right << level)) * kTileM + tt;
+        const unsigned old = atomicExch(node, canonical_bits(part) ^ kNodeKey);
+        if (old == 0u) return;                          // first at the node: the neighbour carries the sum on
+        *node = 0u;                                     // second: empty the node for the next call
+        part += __uint_as_float(old ^ kNodeKey);        // a + b == b + a: the order of arrival does not matter
     }
-    __stcg(p.workspace + (static_cast<int64_t>(blockIdx.x) * 2 + (r != r_first)) * kTileM + tt, part);
-    // The barrier orders the 256 partial sums before thread 0's acq_rel arrival (release: they are
-    // visible to whoever sees the count; acquire: it sees the partials of every earlier arrival), and
-    // the second barrier hands that view to the other 255 threads.
-    asm volatile("bar.sync %0, 256;" ::"r"(bar) : "memory");
-    if (tt == 0) {
-        unsigned old;
-        asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(p.row_counter + r) : "memory");
-        *is_last = (old == static_cast<unsigned>(nseg - 1));
-    }
-    asm volatile("bar.sync %0, 256;" ::"r"(bar) : "memory");
-    if (*is_last) {
-        if (row < p.M) {
-            float sum = 0.f;
-            for (int s = 0; s < nseg; ++s) {
-                const int q = q0 + s;
-                const int slot = (r != static_cast<int>(range_begin(p, q) / static_cast<unsigned>(p.C)));
-                sum += __ldcg(p.workspace + (static_cast<int64_t>(q) * 2 + slot) * kTileM + tt);
-            }
-            store_y(p.y, p.ydt, row, sum);
-        }
-        if (tt == 0) p.row_counter[r] = 0;          // ready for the next call on this handle
-    }
-    asm volatile("bar.sync %0, 256;" ::"r"(bar) : "memory");       // is_last may be rewritten by the next batch
+    store_y(p.y, p.ydt, row, part);
 }
 
 // One persistent CTA per GTile range; every warp runs its own fetch -> decode pipeline.
@@ -286,25 +293,35 @@ spmspv_kernel(const Params p) {
 
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
     const unsigned g_begin = range_begin(p, blockIdx.x), g_end = range_begin(p, blockIdx.x + 1);
-    const int r_first = static_cast<int>(g_begin / static_cast<unsigned>(p.C));
 
     const int lane7 = lane & 7;
     const int lgrp = lane >> 3;
-    const unsigned bit0 = pinned(1u << (4 * lane7));    // first bit of my nibble inside a 32-bit bitmap word
-    const unsigned lt_mask = pinned(bit0 - 1u);
     // fetch role: lane (lgrp, lane7) moves 16-byte pieces lane7, lane7+8, ... and bitmap word lane7 of the
-    // group's lgrp-th tile.  scan role: the same (tile, word).  decode role: nibble lane7 of words w with
-    // (w & 3) == lgrp of every tile of the group.
-    const int tpos = (lane7 & 3) * 8 + lgrp * 2 + (lane7 >> 2);         // where (tile lgrp, word lane7) sits
+    // group's lgrp-th tile.  scan role: the same (tile, word).  decode role: lanes 0-15 take the even
+    // words of every tile, lanes 16-31 the odd ones; a lane owns rows 2*l15, 2*l15+1 of its words, so
+    // the 32 simultaneous value loads of a step fall inside 64 rows = at most 128 contiguous bytes
+    // (one shared-memory wavefront, whatever the density).
+    const int l15 = lane & 15, lhalf = lane >> 4;
+    const unsigned bit0 = pinned(1u << (2 * l15));      // my first row inside a 32-bit bitmap word
+    const unsigned bit1 = pinned(bit0 << 1);
+    const unsigned lt_mask = pinned(bit0 - 1u);
+    const int tpos = (lane7 & 1) * 16 + lgrp * 4 + (lane7 >> 1);        // where (tile lgrp, word lane7) sits
     const uint32_t val_dst = pinned(smem_u32(&sm.ring[warp][0][lgrp * kSlotBytes + 16 * lane7]));
     const uint32_t bm_own = pinned(smem_u32(&sm.tab[warp].bm[0][tpos]));
-    const uint32_t bm_dec = pinned(smem_u32(&sm.tab[warp].bm[0][lgrp * 8]));
-    // voff[i] sits kVoffFromBm - 2*i bytes behind bm[0][i]
-    constexpr uint32_t kVoffFromBm = kDepth * 128;
-    const uint32_t vo_own = bm_own + kVoffFromBm - 2u * tpos;
-    const uint32_t vo_dec = bm_dec + kVoffFromBm - 16u * lgrp;
-    const uint32_t ring_w = pinned(smem_u32(&sm.ring[warp][0][0]));                 // my warp's ring
-    const uint32_t slot_off = pinned(static_cast<uint32_t>(lgrp * kSlotBytes));     // scan role: my tile's slot in a stage
+    const uint32_t bm_dec = pinned(smem_u32(&sm.tab[warp].bm[0][lhalf * 16]));
+    constexpr int kVoFromBm = kDepth * 128;             // vo[d][i] sits this many bytes behind bm[d][i]
+    const uint32_t ring_slot = pinned(smem_u32(&sm.ring[warp][0][lgrp * kSlotBytes]));  // scan role: my tile's slot in stage 0
+    // fetch role: my 16-byte piece of a column tile's values / my bitmap word, before the tile's offset is added
+#if SPDP_PIN_SRC & 1
+    const unsigned char* const val_src = pinned(reinterpret_cast<const unsigned char*>(p.values) + 16 * lane7);
+#else
+    const unsigned char* const val_src = reinterpret_cast<const unsigned char*>(p.values) + 16 * lane7;
+#endif
+#if SPDP_PIN_SRC & 2
+    const unsigned char* const bm_src = pinned(reinterpret_cast<const unsigned char*>(p.bitmap) + 4 * lane7);
+#else
+    const unsigned char* const bm_src = reinterpret_cast<const unsigned char*>(p.bitmap) + 4 * lane7;
+#endif
     const uint32_t rec_addr = smem_u32(&sm.rec[0]);
     const uint32_t x_addr = smem_u32(&sm.xact[0]);
 
@@ -312,7 +329,7 @@ spmspv_kernel(const Params p) {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     bool waited_for_stream = false;  // x, y, workspace and counters may belong to the previous kernel until we wait
 
-    float acc[8];                   // rows 4*lane+k (k<4) and 128+4*lane+(k-4) of the current row tile
+    float acc[8];                   // acc[2s + k] = row 64*s + 2*lane + k of the current row tile
 #pragma unroll
     for (int k = 0; k < 8; ++k) acc[k] = 0.f;
 
@@ -436,10 +453,8 @@ spmspv_kernel(const Params p) {
                 base += __popc(m);
             }
             // null records: the padding in front of piece B and behind the last record
-            if (warp == 0) {
-                if (lane < static_cast<int>(pad)) sm.rec[realA + lane] = make_uint2(0u, kNullRec);
-                if (lane < kGroup) sm.rec[nact + lane] = make_uint2(0u, kNullRec);
-            }
+            if (warp == 0 && lane < static_cast<int>(pad)) sm.rec[realA + lane] = make_uint2(0u, kNullRec);
+            if (t < kRecPad) sm.rec[nact + t] = make_uint2(0u, kNullRec);
         }
         __syncthreads();       // the records are complete; the staging area becomes the ring again
         const int ngroups = (nact + kGroup - 1) / kGroup;
@@ -452,58 +467,68 @@ spmspv_kernel(const Params p) {
         uint32_t dv = 0, db = 0;
         uint32_t rec_nxt = rec_addr + 8u * (warp * kGroup + lgrp);
         // start the copies of group glq (my record at rec_a) into ring position (dv_f, db_f)
-        auto fetch_group = [&](int glq, uint32_t rec_a, uint32_t dv_f, uint32_t db_f) {
-            if (glq < ngroups) {
-                const uint2 rc = lds_v2(rec_a);
-                const uint32_t bdst = bm_own + db_f;
-                if (rc.y != kNullRec) {
-                    const int rem = static_cast<int>(rc.y & 63u) - lane7;                  // my 16-byte pieces left
-                    const unsigned char* src = reinterpret_cast<const unsigned char*>(p.values) + (2 * static_cast<uint64_t>(rc.x) + 16u * lane7);
-                    const uint32_t dst = val_dst + dv_f;
-                    cp_async16<0>(dst, src, rem);
-                    cp_async16<128>(dst, src, rem);
-                    cp_async16<256>(dst, src, rem);
-                    cp_async16<384>(dst, src, rem);
-                    cp_async4(bdst, reinterpret_cast<const unsigned char*>(p.bitmap) + (static_cast<size_t>(rc.y >> 6) * 32 + 4u * lane7));
-                } else {
-                    sts_u32(bdst, 0u);
-                }
+        auto fetch_group = [&](uint32_t rec_a, uint32_t dv_f, uint32_t db_f) {
+            const uint2 rc = lds_v2(rec_a);
+            const uint32_t bdst = bm_own + db_f;
+            if (rc.y != kNullRec) {
+                const int rem = static_cast<int>(rc.y & 63u) - lane7;                  // my 16-byte pieces left
+                const unsigned char* src = offset_wide<2>(val_src, rc.x);
+                const uint32_t dst = val_dst + dv_f;
+                cp_async16<0>(dst, src, rem);
+                cp_async16<128>(dst, src, rem);
+                cp_async16<256>(dst, src, rem);
+                cp_async16<384>(dst, src, rem);
+                cp_async4(bdst, offset_wide<32>(bm_src, rc.y >> 6));
+            } else {
+                sts_u32(bdst, 0u);
             }
             cp_async_commit();
         };
 #pragma unroll
         for (int dd = 0; dd < kDepth; ++dd) {
-            fetch_group(warp + dd * kWarps, rec_nxt, dd * kStageBytes, dd * 128);
+            fetch_group(rec_nxt, dd * kStageBytes, dd * 128);
             rec_nxt += 8u * kGroup * kWarps;
         }
-        const unsigned m1 = pinned(bit0 << 1), m2 = pinned(bit0 << 2), m3 = pinned(bit0 << 3);
         // one group: wait for its copies, scan, decode, refill its ring position with the group kDepth ahead
         auto one_group = [&]() {
             cp_async_wait<kDepth - 1>();
             __syncwarp();
-            {   // scan role: offset of my word's first value inside the warp's ring
-                const unsigned cnt = __popc(lds_u32(bm_own + db));
+            {   // scan role: address of my word's first value inside the warp's ring
+                const uint32_t own = bm_own + db;
+                const unsigned cnt = __popc(lds_u32(own));
                 unsigned inc = cnt;
                 scan8_level<1>(inc);
                 scan8_level<2>(inc);
                 scan8_level<4>(inc);
-                sts_u16(vo_own, slot_off + dv + 2u * (inc - cnt));
+                sts_u32<kVoFromBm>(own, ring_slot + dv + 2u * (inc - cnt));
             }
             __syncwarp();
-            // decode role: my 8 words (tile it, word 4h + lgrp at index 2*it + h), their value offsets, the 4 x
-            const uint32_t x_cur = x_addr + 8u * lq;
+            // decode role: my 16 words (tile it, word 2s + lhalf at index 4*it + s), their value addresses, the 4 x
+            const uint32_t bmd = bm_dec + db;
+            const uint2 xs = lds_v2(x_addr + 8u * lq);
 #pragma unroll 1
-            for (int half = 0; half < 2; ++half) {
-                const uint4 w = lds_v4(bm_dec + db + 16 * half);
-                const uint2 a = lds_v2(vo_dec + 8 * half);                       // four 16-bit offsets
-                const unsigned xs = lds_u32(x_cur + 4 * half);                   // two activations
-                decode_step(w.x, ring_w + (a.x & 0xFFFFu), lt_mask, bit0, m1, m2, m3, xs, acc[0], acc[1], acc[2], acc[3]);
-                decode_step(w.y, ring_w + (a.x >> 16), lt_mask, bit0, m1, m2, m3, xs, acc[4], acc[5], acc[6], acc[7]);
-                decode_step(w.z, ring_w + (a.y & 0xFFFFu), lt_mask, bit0, m1, m2, m3, xs >> 16, acc[0], acc[1], acc[2], acc[3]);
-                decode_step(w.w, ring_w + (a.y >> 16), lt_mask, bit0, m1, m2, m3, xs >> 16, acc[4], acc[5], acc[6], acc[7]);
+            for (int pr = 0; pr < 2; ++pr) {                                     // two column tiles per pass
+                const uint32_t ah = bmd + 32 * pr;
+                const unsigned x2 = pr ? xs.y : xs.x;                            // their two activations
+                {
+                    const uint4 w = lds_v4<0>(ah);
+                    const uint4 a = lds_v4<kVoFromBm>(ah);
+                    decode_step<false>(w.x, a.x, lt_mask, bit0, bit1, x2, acc[0], acc[1]);
+                    decode_step<false>(w.y, a.y, lt_mask, bit0, bit1, x2, acc[2], acc[3]);
+                    decode_step<false>(w.z, a.z, lt_mask, bit0, bit1, x2, acc[4], acc[5]);
+                    decode_step<false>(w.w, a.w, lt_mask, bit0, bit1, x2, acc[6], acc[7]);
+                }
+                {
+                    const uint4 w = lds_v4<16>(ah);
+                    const uint4 a = lds_v4<kVoFromBm + 16>(ah);
+                    decode_step<true>(w.x, a.x, lt_mask, bit0, bit1, x2, acc[0], acc[1]);
+                    decode_step<true>(w.y, a.y, lt_mask, bit0, bit1, x2, acc[2], acc[3]);
+                    decode_step<true>(w.z, a.z, lt_mask, bit0, bit1, x2, acc[4], acc[5]);
+                    decode_step<true>(w.w, a.w, lt_mask, bit0, bit1, x2, acc[6], acc[7]);
+                }
             }
             __syncwarp();                  // everyone is done with this ring position
-            fetch_group(lq + kDepth * kWarps, rec_nxt, dv, db);
+            fetch_group(rec_nxt, dv, db);  // refill it with the group kDepth ahead (null records past the end)
             rec_nxt += 8u * kGroup * kWarps;
             lq += kWarps;
             if (kDepth == 2) {
@@ -516,22 +541,21 @@ spmspv_kernel(const Params p) {
         };
         auto park_first = [&]() {      // my share of the first piece is complete: park it, restart from zero
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                sm.red_first[warp][4 * lane + k] = acc[k];
-                sm.red_first[warp][128 + 4 * lane + k] = acc[4 + k];
-                acc[k] = 0.f;
-                acc[4 + k] = 0.f;
+            for (int q = 0; q < 4; ++q) {
+                *reinterpret_cast<float2*>(&sm.red_first[warp][64 * q + 2 * lane]) = make_float2(acc[2 * q], acc[2 * q + 1]);
+                acc[2 * q] = 0.f;
+                acc[2 * q + 1] = 0.f;
             }
         };
-        bool in_first = (ngtB > 0);
+        int park_at = (ngtB > 0) ? groupsA : 0x7FFFFFFF;      // the first group of piece B (none: never)
         while (lq < ngroups) {
-            if (in_first && lq >= groupsA) {
-                in_first = false;
+            if (lq >= park_at) {
+                park_at = 0x7FFFFFFF;
                 park_first();
             }
             one_group();
         }
-        if (in_first) park_first();
+        if (ngtB > 0 && park_at != 0x7FFFFFFF) park_first();
         cp_async_wait<0>();
         __syncthreads();       // all pipelines drained: the ring is idle
 
@@ -540,11 +564,10 @@ spmspv_kernel(const Params p) {
         const bool done_last = two ? doneB : doneA;             // does the batch's last piece end its row tile here?
         if (done_last) {
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                sm.red[warp][4 * lane + k] = acc[k];            // red[] reuses the idle ring
-                sm.red[warp][128 + 4 * lane + k] = acc[4 + k];
-                acc[k] = 0.f;
-                acc[4 + k] = 0.f;
+            for (int q = 0; q < 4; ++q) {                       // red[] reuses the idle ring
+                *reinterpret_cast<float2*>(&sm.red[warp][64 * q + 2 * lane]) = make_float2(acc[2 * q], acc[2 * q + 1]);
+                acc[2 * q] = 0.f;
+                acc[2 * q + 1] = 0.f;
             }
         }
         __syncthreads();
@@ -552,9 +575,9 @@ spmspv_kernel(const Params p) {
         // batch; the other warps go straight on to the next batch's list phase.  Neither red[] nor
         // red_first[] is written again before these threads have passed the next __syncthreads.
         if (t < kTileM) {
-            if (done_last) finish_row_tile(p, two ? rB : rA, r_first, sm.red, t, 1, &sm.is_last[0]);
+            if (done_last) finish_row_tile(p, two ? rB : rA, sm.red, t);
         } else if (t < 2 * kTileM) {
-            if (two) finish_row_tile(p, rA, r_first, sm.red_first, t - kTileM, 2, &sm.is_last[1]);
+            if (two) finish_row_tile(p, rA, sm.red_first, t - kTileM);
         }
     }
 }
@@ -600,19 +623,17 @@ __global__ void active_columns_kernel(const __half* __restrict__ x, int K, int r
 // tables, the arrival counters, the split-K partial sums) lives here instead, so the entry point
 // below never allocates.  One copy per device that loads the library, held until exit.
 constexpr int kNoAllocMaxCtas = 512;
-constexpr int kNoAllocMaxRowTiles = 4096;          // M <= 1,048,576
 
 struct NoAllocScratch {
-    unsigned row_counter[kNoAllocMaxRowTiles];
     int status;
-    float workspace[kNoAllocMaxCtas * 2 * kTileM];
+    alignas(16) float workspace[kNoAllocMaxCtas * kTileM];
 };
 
 static __device__ __align__(256) unsigned char g_noalloc_scratch[sizeof(NoAllocScratch)];
 
-// Zeroes what a call expects to start at zero (the array keeps whatever the previous call left).
-__global__ void noalloc_setup_kernel(NoAllocScratch* sc, int R) {
-    for (int r = blockIdx.x * blockDim.x + threadIdx.x; r < R; r += gridDim.x * blockDim.x) sc->row_counter[r] = 0;
+// Empties what a call expects to find empty (the array keeps whatever an aborted call left).
+__global__ void noalloc_setup_kernel(NoAllocScratch* sc, int words) {
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < words; i += gridDim.x * blockDim.x) sc->workspace[i] = 0.f;
     if (blockIdx.x == 0 && threadIdx.x == 0) sc->status = 0;
 }
 
@@ -657,7 +678,6 @@ spdp_status launch_spmspv(const spdp_matrix* h, const __half* x, int rule, float
     p.NGT = h->NGT;
     p.num_ctas = h->num_ctas;
     p.workspace = h->workspace;
-    p.row_counter = h->row_counter;
     p.status = h->status_word;
     return launch_kernel(p, h->num_ctas, s);
 }
@@ -670,7 +690,7 @@ spdp_status launch_spmspv_noalloc(const uint32_t* tileoffset, const uint32_t* co
     static int sm_count_of[kMaxDevices] = {};
     static std::mutex mu;
     const int64_t R = (M + kTileM - 1) / kTileM, C = (K + kTileK - 1) / kTileK, NGT = R * C;
-    if (R > kNoAllocMaxRowTiles || NGT * kTileK >= (int64_t(1) << 26)) return SPDP_ERR_UNSUPPORTED_SHAPE;
+    if (NGT * kTileK >= (int64_t(1) << 26)) return SPDP_ERR_UNSUPPORTED_SHAPE;
     int dev = 0;
     SPDP_CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= kMaxDevices) return SPDP_ERR_UNSUPPORTED_SHAPE;
@@ -691,7 +711,7 @@ spdp_status launch_spmspv_noalloc(const uint32_t* tileoffset, const uint32_t* co
     }
     int P = sms * kCtasPerSm < kNoAllocMaxCtas ? sms * kCtasPerSm : kNoAllocMaxCtas;
     if (P > NGT) P = static_cast<int>(NGT);
-    noalloc_setup_kernel<<<(static_cast<int>(R) + 255) / 256, 256, 0, s>>>(sc, static_cast<int>(R));
+    noalloc_setup_kernel<<<(P * kTileM + 1023) / 1024, 256, 0, s>>>(sc, P * kTileM);
     SPDP_CUDA_TRY(cudaGetLastError());
     Params p;
     p.tileoffset = tileoffset;
@@ -711,7 +731,6 @@ spdp_status launch_spmspv_noalloc(const uint32_t* tileoffset, const uint32_t* co
     p.NGT = NGT;
     p.num_ctas = P;
     p.workspace = sc->workspace;            // addresses inside the device array (no host dereference)
-    p.row_counter = sc->row_counter;
     p.status = &sc->status;
     return launch_kernel(p, P, s);
 }

@@ -62,8 +62,8 @@ def test_noalloc_rejects_oversize_and_bad_arguments(S):
     x = torch.zeros(16, dtype=torch.float16, device="cuda")
     y = torch.zeros(16, dtype=torch.float32, device="cuda")
     buf = torch.zeros(64, dtype=torch.int64, device="cuda")
-    with pytest.raises(S.SpdpError, match="UNSUPPORTED_SHAPE"):       # more than 4096 row tiles
-        S.spdp_spmspv_noalloc(buf, buf, buf, buf, 4097 * 256, 16, x, 0, 0.0, y)
+    with pytest.raises(S.SpdpError, match="UNSUPPORTED_SHAPE"):       # 2^26 column tiles: beyond the library's limit
+        S.spdp_spmspv_noalloc(buf, buf, buf, buf, (1 << 22) * 256, 16, x, 0, 0.0, y)
     with pytest.raises(S.SpdpError, match="INVALID_ARG"):
         S.spdp_spmspv_noalloc(buf, buf, buf, buf, 16, 16, x, 2, 0.0, y)      # mask rule without a mask
     with pytest.raises(S.SpdpError, match="INVALID_ARG"):

@@ -33,11 +33,9 @@ namespace {
 #ifndef SPDP_DEPTH
 #define SPDP_DEPTH 2
 #endif
-#ifndef SPDP_PIN_SRC
-#define SPDP_PIN_SRC 3
-#endif
-#ifndef SPDP_UNROLL_HALF
-#define SPDP_UNROLL_HALF 0
+#ifndef SPDP_L2HINT
+#define SPDP_L2HINT ".L2::64B"   // fill granularity asked of L2 for the value / bitmap copies: a column tile is a
+                                 // few hundred bytes between skipped neighbours, so whole 128-byte lines over-fetch
 #endif
 constexpr int kWarps = SPDP_WARPS;         // warps per CTA; every warp fetches and decodes its own column tiles
 constexpr int kDepth = SPDP_DEPTH;         // groups a warp keeps in flight
@@ -49,7 +47,7 @@ constexpr int kThreads = kWarps * 32;
 constexpr int kChunkCols = SPDP_CHUNK_COLS; // columns handled between two pipeline drains
 constexpr int kCtasPerSm = SPDP_CTAS_PER_SM;
 constexpr uint32_t kNullRec = 0xFFFFFFFFu;
-constexpr int kMaxGroupsPerWarp = (kChunkCols / 32 + kWarps - 1) / kWarps;   // 32-position groups a warp lists per batch
+constexpr int kListPasses = (kChunkCols / 8 + kThreads - 1) / kThreads;     // 8-position units a thread lists per batch
 constexpr int kChunkGT = kChunkCols / kTileK;
 constexpr int kRecPad = kGroup * (kDepth * kWarps + 1);   // null records behind the last real one
 
@@ -96,7 +94,7 @@ struct __align__(128) Smem {
                                                         //      can fetch kDepth groups ahead without a range test
     alignas(16) unsigned short xact[kChunkCols + kGroup];   // its activation x_j (fp16 bits)
     float red_first[kWarps][kTileM];                    // row reduction of a batch's first piece (flushed mid-stream)
-    uint32_t warp_total[kWarps][2];                     // list phase: records listed by each warp (all, piece A)
+    uint32_t warp_total[kListPasses][kWarps][2];        // list phase: records listed by each warp per pass (all, piece A)
 };
 static_assert(offsetof(Smem, rec) % 16 == 0 && offsetof(Smem, xact) % 16 == 0 && offsetof(Smem, tab) % 16 == 0, "16-byte shared loads need aligned tables");
 static_assert(sizeof(float) * kWarps * kTileM <= size_t(kWarps) * kDepth * kStageBytes, "red must fit in the ring");
@@ -133,7 +131,7 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) {
 // Asynchronous global -> shared copies (Sec. 4.2.3: 128-bit per thread); `on` = false copies nothing.
 template <int kOff>
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int rem) {
-    asm volatile("{\n .reg .pred p;\n setp.gt.s32 p, %2, %3;\n @p cp.async.cg.shared.global [%0+%4], [%1+%4], 16;\n}"
+    asm volatile("{\n .reg .pred p;\n setp.gt.s32 p, %2, %3;\n @p cp.async.cg.shared.global" SPDP_L2HINT " [%0+%4], [%1+%4], 16;\n}"
                  ::"r"(dst), "l"(src), "r"(rem), "n"(kOff / 16), "n"(kOff) : "memory");
 }
 // 16-byte copy that reads only the first `bytes` (0..16) source bytes and zero-fills the rest.
@@ -141,7 +139,7 @@ __device__ __forceinline__ void cp_async16_partial(uint32_t dst, const void* src
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ void cp_async4(uint32_t dst, const void* src) {
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
+    asm volatile("cp.async.ca.shared.global" SPDP_L2HINT " [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
@@ -276,12 +274,13 @@ __device__ __forceinline__ void finish_row_tile(const Params& p, int r, const fl
 // that the usual CTA range (the tail of one row tile and the head of the next) is one batch.
 // Per batch:
 //   (1) all warps: the pieces' ColInfo / TileOffset words and the active-column list from x
-//       (ballots + prefix sums), one record per active column tile -- Sec. 4.2 steps (1)-(3);
+//       (a thread tests 8 columns, warp scans + prefix sums place them), one record per active
+//       column tile -- Sec. 4.2 steps (1)-(3);
 //   (2) each warp takes groups of kGroup active column tiles round-robin.  It keeps kDepth
 //       groups in flight: the padded values of a column tile arrive with 16-byte asynchronous
 //       copies (lane = one 16-byte piece of one of the group's tiles), its 8 bitmap words with
-//       4-byte ones; inactive columns are never touched.  Decode (Sec. 4.2.1): lane owns 4
-//       consecutive rows of a half column tile, rank = set bits before them, values read from
+//       4-byte ones; inactive columns are never touched.  Decode (Sec. 4.2.1): lane owns 2
+//       consecutive rows of every second bitmap word, rank = set bits before them, values read from
 //       shared memory, fp32 accumulation in registers.  Where the first piece's groups end the
 //       warp parks its sums in shared memory and starts the second piece from zero;
 //   (3) batch end: cross-warp row reduction, split-K combine and store of every row tile that
@@ -312,16 +311,8 @@ spmspv_kernel(const Params p) {
     constexpr int kVoFromBm = kDepth * 128;             // vo[d][i] sits this many bytes behind bm[d][i]
     const uint32_t ring_slot = pinned(smem_u32(&sm.ring[warp][0][lgrp * kSlotBytes]));  // scan role: my tile's slot in stage 0
     // fetch role: my 16-byte piece of a column tile's values / my bitmap word, before the tile's offset is added
-#if SPDP_PIN_SRC & 1
     const unsigned char* const val_src = pinned(reinterpret_cast<const unsigned char*>(p.values) + 16 * lane7);
-#else
-    const unsigned char* const val_src = reinterpret_cast<const unsigned char*>(p.values) + 16 * lane7;
-#endif
-#if SPDP_PIN_SRC & 2
     const unsigned char* const bm_src = pinned(reinterpret_cast<const unsigned char*>(p.bitmap) + 4 * lane7);
-#else
-    const unsigned char* const bm_src = reinterpret_cast<const unsigned char*>(p.bitmap) + 4 * lane7;
-#endif
     const uint32_t rec_addr = smem_u32(&sm.rec[0]);
     const uint32_t x_addr = smem_u32(&sm.xact[0]);
 
@@ -359,8 +350,6 @@ spmspv_kernel(const Params p) {
         g0 += ngtB;
         const int rB = rA + 1;
         const int nlist = (ngtB > 0) ? vB0 + nB : nA;               // list positions (A, padding, B)
-        const int ngroups32 = (nlist + 31) >> 5;
-        const int qB = (ngtB > 0) ? (vB0 >> 5) : ngroups32;         // first 32-position group of piece B
 
         // ---- (1) active-column list of the batch (ballots + prefix sums) and its records ----
         // One memory round trip: the pieces' ColInfo and TileOffset words and their slice of x stream
@@ -395,62 +384,91 @@ spmspv_kernel(const Params p) {
         }
         cp_async_wait<0>();
         __syncthreads();
-        // Warp w lists the 32-position groups [w * gpw, (w + 1) * gpw): one ballot per group, kept in
-        // registers; the warps' totals meet in shared memory, every warp derives its first record index
+        // A thread lists 8 consecutive positions per pass (unit (pass * kThreads + t)): the DP test on its
+        // 8 activations gives an 8-bit mask, a warp scan of the counts its place among the warp's
+        // records; the warps' totals meet in shared memory, every thread derives its first record index
         // from them, and the records are written in list order.  Piece B starts on a whole group of
         // kGroup records: the padding is inserted in front of its first record.
-        const int gpw = (ngroups32 + kWarps - 1) / kWarps;
-        unsigned masks[kMaxGroupsPerWarp];
-        {
-            unsigned tot = 0, totA = 0;
+        unsigned m8[kListPasses], below[kListPasses];
 #pragma unroll
-            for (int k = 0; k < kMaxGroupsPerWarp; ++k) {
-                const int q = warp * gpw + k;
-                const int v = q * 32 + lane;                             // list position
-                const int j = (v < vB0) ? jA0 + v : v - vB0;             // its column
-                bool a = (k < gpw) && ((v < vB0) ? (v < nA) : (v < nlist));
-                if (a) {
-                    if (p.rule == SPDP_DP_ABS_GT)
-                        a = !(fabsf(__half2float(__ushort_as_half(sm.stage.x[v]))) <= p.thr);
-                    else if (p.rule == SPDP_DP_MASK)
-                        a = (__ldg(p.mask + (j >> 5)) >> (j & 31)) & 1u;
+        for (int k = 0; k < kListPasses; ++k) {
+            const int v0 = (k * kThreads + t) * 8;                       // first list position of my unit
+            unsigned m = 0;
+            if (v0 < nlist) {
+                const int lim = ((v0 < vB0) ? nA : nlist) - v0;          // positions of the unit that hold a column
+                if (p.rule == SPDP_DP_ABS_GT) {
+                    const uint4 xv = *reinterpret_cast<const uint4*>(&sm.stage.x[v0]);
+                    const unsigned xw[4] = {xv.x, xv.y, xv.z, xv.w};
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const float lo = __half2float(__ushort_as_half(static_cast<unsigned short>(xw[i] & 0xFFFFu)));
+                        const float hi = __half2float(__ushort_as_half(static_cast<unsigned short>(xw[i] >> 16)));
+                        m |= (!(fabsf(lo) <= p.thr) ? 1u : 0u) << (2 * i);
+                        m |= (!(fabsf(hi) <= p.thr) ? 1u : 0u) << (2 * i + 1);
+                    }
+                } else if (p.rule == SPDP_DP_MASK) {
+                    const int j0 = (v0 < vB0) ? jA0 + v0 : v0 - vB0;     // a multiple of 8
+                    m = (__ldg(p.mask + (j0 >> 5)) >> (j0 & 31)) & 0xFFu;
+                } else {
+                    m = 0xFFu;
                 }
-                masks[k] = __ballot_sync(0xFFFFFFFFu, a);
-                const unsigned c = __popc(masks[k]);
-                tot += c;
-                if (q < qB) totA += c;
+                m &= (lim >= 8) ? 0xFFu : (lim > 0 ? (1u << lim) - 1u : 0u);
             }
-            if (lane == 0) {
-                sm.warp_total[warp][0] = tot;
-                sm.warp_total[warp][1] = totA;
+            m8[k] = m;
+            const unsigned c = __popc(m);
+            unsigned inc = c;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const unsigned u = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+                if (lane >= d) inc += u;
+            }
+            below[k] = inc - c;
+            const unsigned totA = __reduce_add_sync(0xFFFFFFFFu, (v0 < vB0) ? c : 0u);
+            if (lane == 31) {
+                sm.warp_total[k][warp][0] = inc;
+                sm.warp_total[k][warp][1] = totA;
             }
         }
         __syncthreads();
         int nact, nactA_pad;
         {
-            const unsigned tl = (lane < kWarps) ? sm.warp_total[lane][0] : 0u;
-            const unsigned tla = (lane < kWarps) ? sm.warp_total[lane][1] : 0u;
-            const unsigned realA = __reduce_add_sync(0xFFFFFFFFu, tla);                     // records of piece A
+            unsigned base[kListPasses], total = 0, realA = 0;
+#pragma unroll
+            for (int k = 0; k < kListPasses; ++k) {
+                const unsigned tl = (lane < kWarps) ? sm.warp_total[k][lane][0] : 0u;
+                const unsigned tla = (lane < kWarps) ? sm.warp_total[k][lane][1] : 0u;
+                base[k] = total + __reduce_add_sync(0xFFFFFFFFu, lane < warp ? tl : 0u);   // before my warp's unit run
+                total += __reduce_add_sync(0xFFFFFFFFu, tl);
+                realA += __reduce_add_sync(0xFFFFFFFFu, tla);                             // records of piece A
+            }
             const unsigned pad = (ngtB > 0) ? (kGroup - realA % kGroup) % kGroup : 0u;
-            const unsigned total = __reduce_add_sync(0xFFFFFFFFu, tl) + pad;
-            unsigned base = __reduce_add_sync(0xFFFFFFFFu, lane < warp ? tl : 0u);          // before my first group
+            total += pad;
             nact = static_cast<int>(total);
             nactA_pad = (ngtB > 0) ? static_cast<int>(realA + pad) : ((nact + kGroup - 1) / kGroup) * kGroup;
             const unsigned slotA0 = gA * kTileK - jA0, slotB0 = gB * kTileK;                 // column slot of column 0
 #pragma unroll
-            for (int k = 0; k < kMaxGroupsPerWarp; ++k) {
-                const int q = warp * gpw + k;
-                const unsigned m = masks[k];
-                if ((m >> lane) & 1u) {
-                    const int v = q * 32 + lane;
-                    const int j = (v < vB0) ? jA0 + v : v - vB0;
-                    const unsigned slot = (v < vB0 ? slotA0 : slotB0) + j;
-                    const int item = static_cast<int>(base + (q >= qB ? pad : 0u) + __popc(m & ((1u << lane) - 1u)));
-                    const uint32_t ci = sm.stage.colinfo[v];                                // ColInfo: offset << 16 | nnz
-                    sm.rec[item] = make_uint2(sm.stage.tileoff[v >> 4] + (ci >> 16), (slot << 6) | (((ci & 0xFFFFu) + 7u) >> 3));
-                    sm.xact[item] = sm.stage.x[v];
+            for (int k = 0; k < kListPasses; ++k) {
+                const unsigned m = m8[k];
+                if (m != 0u) {
+                    const int v0 = (k * kThreads + t) * 8;
+                    const bool inB = v0 >= vB0;
+                    const unsigned slot0 = inB ? slotB0 + (v0 - vB0) : slotA0 + jA0 + v0;   // column slot of position v0
+                    int item = static_cast<int>(base[k] + (inB ? pad : 0u) + below[k]);
+                    const unsigned to = sm.stage.tileoff[v0 >> 4];
+                    const uint4 xv = *reinterpret_cast<const uint4*>(&sm.stage.x[v0]);
+                    const uint4 c0 = *reinterpret_cast<const uint4*>(&sm.stage.colinfo[v0]);
+                    const uint4 c1 = *reinterpret_cast<const uint4*>(&sm.stage.colinfo[v0 + 4]);
+                    const unsigned xw[4] = {xv.x, xv.y, xv.z, xv.w};
+                    const unsigned ci[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};   // ColInfo: offset << 16 | nnz
+#pragma unroll
+                    for (int b = 0; b < 8; ++b) {
+                        if ((m >> b) & 1u) {
+                            sm.rec[item] = make_uint2(to + (ci[b] >> 16), ((slot0 + b) << 6) | (((ci[b] & 0xFFFFu) + 7u) >> 3));
+                            sm.xact[item] = static_cast<unsigned short>((b & 1) ? (xw[b >> 1] >> 16) : (xw[b >> 1] & 0xFFFFu));
+                            ++item;
+                        }
+                    }
                 }
-                base += __popc(m);
             }
             // null records: the padding in front of piece B and behind the last record
             if (warp == 0 && lane < static_cast<int>(pad)) sm.rec[realA + lane] = make_uint2(0u, kNullRec);

@@ -141,8 +141,11 @@ class ClockSampler:
                 "window": "timed" if use is self.timed_samples else "warmup+timed"}
 
 
-def cpu_baseline(w, B_active_full):
-    """The C oracle as it stands on the host cores: best of 3 full calls of the same workload."""
+def cpu_baseline(w, B_active_full, gpu=None):
+    """The C oracle as it stands on the host cores: best of 3 full calls of the same workload,
+    one call on one thread, and (with `gpu` = what the CUDA path produced for this workload) how
+    far the CUDA path is from it: packed arrays and active set bit for bit, y against the bound
+    |y - y_ref| <= 1e-3 * sum|W x| + 1e-5."""
     from oracle import c_oracle
     a = c_oracle.active(w.x, w.rule, w.thr)
     best = float("inf")
@@ -154,8 +157,26 @@ def cpu_baseline(w, B_active_full):
         best = min(best, time.perf_counter() - t0)
         if time.perf_counter() - t_total > 30:
             break
-    return {"value": B_active_full / best / 1e9, "unit": UNIT, "cores": used, "kind": "oracle",
-            "sample": f"whole {w.name} call (fp64 dense masked W), best of 3", "ms_per_call": best * 1e3}
+    out = {"value": B_active_full / best / 1e9, "unit": UNIT, "cores": used, "kind": "oracle",
+           "sample": f"whole {w.name} call (fp64 dense masked W), best of 3", "ms_per_call": best * 1e3}
+    t0 = time.perf_counter()
+    y_ref, S, _ = c_oracle.spmspv(w.W, w.x, a, threads=1, want_scale=True)
+    out["ms_per_call_1_thread"] = (time.perf_counter() - t0) * 1e3
+    if gpu is not None:
+        err = np.abs(gpu["y"].astype(np.float64) - y_ref)
+        bound = 1e-3 * S + 1e-5
+        pk = c_oracle.pack(w.W)
+        words = np.zeros((w.K + 31) // 32 * 32, dtype=np.uint8)
+        words[:w.K] = np.asarray(a, dtype=np.uint8)
+        a_words = np.packbits(words, bitorder="little").view(np.uint32)
+        out["parity"] = {
+            "max_normalised_error": float(np.max(err / bound)),
+            "format_equal": bool(all(np.array_equal(np.asarray(pk[k]).view(np.uint8).reshape(-1),
+                                                    np.asarray(gpu["packed"][k]).view(np.uint8).reshape(-1))
+                                     for k in ("tileoffset", "colinfo", "bitmap", "values"))),
+            "active_set_equal": bool(np.array_equal(a_words, gpu["active_words"])),
+        }
+    return out
 
 
 def run_reference(args):
@@ -200,6 +221,7 @@ def main():
     ap.add_argument("--num-ctas", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-context", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay timing")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -235,7 +257,8 @@ def main():
     torch.cuda.synchronize()
     active_words = words.cpu().numpy().view(np.uint32)
     n_active = int(np.unpackbits(active_words.view(np.uint8)).sum())
-    B_active = active_bytes(spdp.spdp_export(h0)["colinfo"], active_words, w.M, w.K, 2)
+    packed_gpu = spdp.spdp_export(h0)
+    B_active = active_bytes(packed_gpu["colinfo"], active_words, w.M, w.K, 2)
     copies = args.copies or max(2, int(np.ceil(2 * l2 / B_active)) + 1)
     handles = [h0] + [spdp.spdp_pack_tiled_cbc(Wd) for _ in range(copies - 1)]
     if args.num_ctas:
@@ -272,6 +295,38 @@ def main():
     ms = max_over_ranks(ms, world)
     ms_per_step = ms / args.steps
     value = replica_value(B_active, world, ms_per_step)
+
+    y_gpu = ys[0].float().cpu().numpy()
+
+    # ---- the same calls replayed from a CUDA graph (launch overhead out of the picture) ----
+    graph_stats = None
+    if not args.no_graph:
+        calls = copies * max(1, -(-100 // copies))              # >= 100 calls, whole rotations
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            for i in range(copies):
+                step(i)
+            side.synchronize()
+            with torch.cuda.graph(g, stream=side):
+                for i in range(calls):
+                    step(i)
+            for _ in range(10):
+                g.replay()
+            side.synchronize()
+            per_call = []
+            for _ in range(10):
+                g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                g0.record(side)
+                g.replay()
+                g1.record(side)
+                side.synchronize()
+                per_call.append(g0.elapsed_time(g1) / calls * 1e3)
+        torch.cuda.current_stream().wait_stream(side)
+        graph_stats = {"calls_per_graph": calls, "replays": 10, "us_per_call_min": min(per_call),
+                       "us_per_call_median": float(np.median(per_call)), "us_per_call_max": max(per_call)}
+        del g
 
     # ---- end to end through the host-vector entry point ----------------------------------
     xh = torch.from_numpy(w.x.copy()).pin_memory()
@@ -334,6 +389,7 @@ def main():
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(2 * w.K),
                 "d2h_bytes_per_step": int(2 * w.M), "us_per_call": e2e_s / e2e_steps * 1e6, "steps": e2e_steps},
         "gpu_launches": args.steps,
+        "graph": graph_stats,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_kind": f"of {peak_kind}", "traffic": NCU_TRAFFIC_BYTES.get(args.workload),
                      "kernel": "spmspv_kernel", "algorithmic_bytes": int(B_active),
@@ -342,7 +398,8 @@ def main():
                     "ideal_speedup_over_dense": 2 * w.M * w.K / B_active},
     }
     if not args.no_cpu_baseline:
-        out["cpu_baseline"] = cpu_baseline(w, B_active)
+        out["cpu_baseline"] = cpu_baseline(w, B_active, {"y": y_gpu, "packed": packed_gpu,
+                                                         "active_words": active_words})
     for h in handles:
         spdp.spdp_free(h)
     print(json.dumps(out))

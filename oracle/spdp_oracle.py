@@ -290,6 +290,35 @@ def spmspv_bruteforce(W, x, active):
     return y, S
 
 
+def spmspv_batch_ref(W, X, actives):
+    """Small-batch decode (the paper's future work, Sec. 6): B tokens share one pass over W_sp and
+    every token keeps its own active set.  The result is the single-vector definition of Sec. 4.2
+    applied token by token: Y[b][i] = sum_{j in A_b} W[i][j] * X[b][j], S[b][i] the matching error
+    scale.  X is [B][K], actives is [B][K] bool.  Returns (Y, S), float64 [B][M]."""
+    X = np.asarray(X)
+    actives = np.asarray(actives, dtype=bool)
+    ys, ss = [], []
+    for b in range(X.shape[0]):
+        y, S = spmspv_ref(W, X[b], actives[b])
+        ys.append(y)
+        ss.append(S)
+    return np.stack(ys), np.stack(ss)
+
+
+def union_active(actives) -> np.ndarray:
+    """Columns that at least one token of the batch keeps: what a batched call has to fetch."""
+    return np.asarray(actives, dtype=bool).any(axis=0)
+
+
+def active_bytes_batch(p: dict, actives, y_bytes_per_elem: int = 2) -> int:
+    """Bytes a batched call must move: the matrix bytes of the union of the tokens' active columns
+    (once), and every token's x and y."""
+    actives = np.asarray(actives, dtype=bool)
+    B = actives.shape[0]
+    one = active_bytes(p, union_active(actives), y_bytes_per_elem)
+    return one + (B - 1) * (2 * p["K"] + y_bytes_per_elem * p["M"])
+
+
 def tolerance(S) -> np.ndarray:
     """Per-output bound of the parity gate: 1e-3 * S[i] + 1e-5."""
     return 1e-3 * np.asarray(S, dtype=np.float64) + 1e-5

@@ -14,9 +14,12 @@
 #include <mutex>
 
 #include "spdp_internal.h"
+#include "spmspv_device.cuh"
 
 namespace spdp {
 namespace {
+
+using namespace dev;
 
 #ifndef SPDP_FMA_MODE
 #define SPDP_FMA_MODE 0      // 0: mixed-precision fma.rn.f32.f16, 1: cvt + fp32 fma
@@ -32,10 +35,6 @@ namespace {
 #endif
 #ifndef SPDP_DEPTH
 #define SPDP_DEPTH 2
-#endif
-#ifndef SPDP_L2HINT
-#define SPDP_L2HINT ".L2::64B"   // fill granularity asked of L2 for the value / bitmap copies: a column tile is a
-                                 // few hundred bytes between skipped neighbours, so whole 128-byte lines over-fetch
 #endif
 constexpr int kWarps = SPDP_WARPS;         // warps per CTA; every warp fetches and decodes its own column tiles
 constexpr int kDepth = SPDP_DEPTH;         // groups a warp keeps in flight
@@ -112,39 +111,6 @@ __device__ __forceinline__ bool column_active(int rule, float thr, const uint32_
     return (mask[j >> 5] >> (j & 31)) & 1u;
 }
 
-__device__ __forceinline__ void store_y(void* y, int ydt, int64_t i, float v) {
-    if (ydt == SPDP_Y_F32) static_cast<float*>(y)[i] = v;
-    else static_cast<__half*>(y)[i] = __float2half_rn(v);
-}
-
-// Makes a loop-invariant value opaque to the compiler, so that it stays in its register instead of
-// being recomputed from the thread index inside the hot loop.
-template <typename T>
-__device__ __forceinline__ T pinned(T v) {
-    if constexpr (sizeof(T) == 8) asm volatile("" : "+l"(v));
-    else asm volatile("" : "+r"(v));
-    return v;
-}
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-// Asynchronous global -> shared copies (Sec. 4.2.3: 128-bit per thread); `on` = false copies nothing.
-template <int kOff>
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, int rem) {
-    asm volatile("{\n .reg .pred p;\n setp.gt.s32 p, %2, %3;\n @p cp.async.cg.shared.global" SPDP_L2HINT " [%0+%4], [%1+%4], 16;\n}"
-                 ::"r"(dst), "l"(src), "r"(rem), "n"(kOff / 16), "n"(kOff) : "memory");
-}
-// 16-byte copy that reads only the first `bytes` (0..16) source bytes and zero-fills the rest.
-__device__ __forceinline__ void cp_async16_partial(uint32_t dst, const void* src, int bytes) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void cp_async4(uint32_t dst, const void* src) {
-    asm volatile("cp.async.ca.shared.global" SPDP_L2HINT " [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-
 // One decode step (Sec. 4.2.1): the 2 consecutive rows this lane owns inside the 32-bit bitmap
 // word W.  `first` is the shared-memory address of the word's first value, `below` masks the bits
 // of lower rows, m0 and m1 are the lane's two bits.  rank = set bits before the position; a set
@@ -188,64 +154,17 @@ __device__ __forceinline__ void decode_step(unsigned W, uint32_t first, unsigned
         asm volatile(SPDP_DECODE_BODY("xl")
                      : "+f"(a0), "+f"(a1) : "r"(W), "r"(first), "r"(below), "r"(m0), "r"(m1), "r"(x32));
 }
-// One level of an inclusive prefix sum over segments of 8 lanes.
-template <int kDelta>
-__device__ __forceinline__ void scan8_level(unsigned& v) {
-    asm volatile("{\n .reg .pred p;\n .reg .b32 u;\n shfl.sync.up.b32 u|p, %0, %1, 0x1800, 0xffffffff;\n @p add.u32 %0, %0, u;\n}"
-                 : "+r"(v) : "n"(kDelta));
-}
-__device__ __forceinline__ unsigned lds_u32(uint32_t addr) {
-    unsigned v;
-    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
-    return v;
-}
-template <int kOff>
-__device__ __forceinline__ uint4 lds_v4(uint32_t addr) {
-    uint4 v;
-    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4+%5];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr), "n"(kOff));
-    return v;
-}
-__device__ __forceinline__ uint2 lds_v2(uint32_t addr) {
-    uint2 v;
-    asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
-    return v;
-}
-template <int kOff = 0>
-__device__ __forceinline__ void sts_u32(uint32_t addr, unsigned v) {
-    asm volatile("st.shared.u32 [%0+%2], %1;" ::"r"(addr), "r"(v), "n"(kOff) : "memory");
-}
-// base + a * kScale with a 64-bit result (one multiply-add)
-template <int kScale>
-__device__ __forceinline__ const unsigned char* offset_wide(const unsigned char* base, uint32_t a) {
-    const unsigned char* r;
-    asm("mad.wide.u32 %0, %1, %2, %3;" : "=l"(r) : "r"(a), "n"(kScale), "l"(base));
-    return r;
-}
-
-// The work split: CTA c owns GTiles [range_begin(c), range_begin(c + 1)) of the row-major GTile order.
-// NGT < 2^22 and num_ctas <= 1024 keep every product below 2^32.
 __device__ __forceinline__ unsigned range_begin(const Params& p, unsigned c) {
-    return (static_cast<unsigned>(p.NGT) * c) / static_cast<unsigned>(p.num_ctas);
+    return dev::range_begin(static_cast<unsigned>(p.NGT), static_cast<unsigned>(p.num_ctas), c);
 }
-// The CTA whose range holds GTile g: ceil((g + 1) * num_ctas / NGT) - 1.
 __device__ __forceinline__ int range_owner(const Params& p, unsigned g) {
-    const unsigned ngt = static_cast<unsigned>(p.NGT);
-    return static_cast<int>(((g + 1u) * static_cast<unsigned>(p.num_ctas) + ngt - 1u) / ngt) - 1;
+    return dev::range_owner(static_cast<unsigned>(p.NGT), static_cast<unsigned>(p.num_ctas), g);
 }
-
-// A partial sum is kept in the workspace XOR this key, so that the all-zero word means "empty".
-// NaN sums are made canonical first, which keeps a stored word from ever being zero.
-constexpr unsigned kNodeKey = 0xFFC0DEADu;
-__device__ __forceinline__ unsigned canonical_bits(float v) { return (v != v) ? 0x7FFFFFFFu : __float_as_uint(v); }
 
 // Adds the kWarps per-warp partial sums of one row tile in warp order and finishes the row (tt =
 // row inside the tile; the rows are independent, nothing here synchronises threads).  A row tile
-// fed by one segment is stored directly.  Otherwise segment i of the row tile's nseg segments is
-// leaf i of a binary tree: at level l, node idx stands for segments [idx << l, (idx + 1) << l); a
-// node without a right-hand neighbour moves up unchanged.  The meeting place of nodes (idx, idx | 1)
-// is the workspace row of the CTA that owns the right node's first segment -- a CTA that starts
-// inside this row tile, and a different one for every tree node.
+// fed by one segment is stored directly; otherwise the segments' sums meet along the fixed tree of
+// tree_combine and the thread that completes the root stores y.
 __device__ __forceinline__ void finish_row_tile(const Params& p, int r, const float (*red)[kTileM], int tt) {
     float part = 0.f;
 #pragma unroll
@@ -254,18 +173,9 @@ __device__ __forceinline__ void finish_row_tile(const Params& p, int r, const fl
     if (row >= p.M) return;
     const int q0 = range_owner(p, static_cast<unsigned>(r) * p.C);                 // first and last CTA feeding row tile r
     const int nseg = range_owner(p, static_cast<unsigned>(r + 1) * p.C - 1u) - q0 + 1;
-    int idx = static_cast<int>(blockIdx.x) - q0;
-    for (int n = nseg, level = 0; n > 1; n = (n + 1) >> 1, ++level, idx >>= 1) {
-        const int right = idx | 1;
-        if (right >= n) continue;                       // no neighbour at this level
-        unsigned* node = reinterpret_cast<unsigned*>(p.workspace) +
-                         static_cast<int64_t>(q0 + (right << level)) * kTileM + tt;
-        const unsigned old = atomicExch(node, canonical_bits(part) ^ kNodeKey);
-        if (old == 0u) return;                          // first at the node: the neighbour carries the sum on
-        *node = 0u;                                     // second: empty the node for the next call
-        part += __uint_as_float(old ^ kNodeKey);        // a + b == b + a: the order of arrival does not matter
-    }
-    store_y(p.y, p.ydt, row, part);
+    if (tree_combine(part, reinterpret_cast<unsigned*>(p.workspace) + tt, kTileM, q0, nseg,
+                     static_cast<int>(blockIdx.x) - q0))
+        store_y(p.y, p.ydt, row, part);
 }
 
 // One persistent CTA per GTile range; every warp runs its own fetch -> decode pipeline.

@@ -144,3 +144,49 @@ def test_result_from_packed_equals_result_from_dense():
     y, _ = O.spmspv_ref(W, x, a)
     y2, _ = O.spmspv_ref(O.unpack_ref(O.pack_ref(W)), x, a)
     assert np.array_equal(y, y2)
+
+
+# ------------------------------------------------------------------------------------------
+# small-batch definition (Sec. 6, future work): the single-vector definition token by token
+# ------------------------------------------------------------------------------------------
+def test_batch_dense_special_case_is_a_matrix_product():
+    """No pruning of either kind: Y = X W^T, checked against NumPy's matmul."""
+    rng = np.random.Generator(np.random.PCG64(71))
+    M, K, B = 300, 200, 5
+    W = (rng.standard_normal((M, K)) * 0.05).astype(np.float16)
+    X = rng.standard_normal((B, K)).astype(np.float16)
+    Y, S = O.spmspv_batch_ref(W, X, np.ones((B, K), bool))
+    assert np.allclose(Y, X.astype(np.float64) @ W.astype(np.float64).T, rtol=1e-12, atol=1e-12)
+    assert np.all(S >= np.abs(Y) - 1e-12)
+
+
+def test_batch_is_brute_force_per_token_and_follows_token_order():
+    rng = np.random.Generator(np.random.PCG64(72))
+    M, K, B = 40, 50, 3
+    W = rng.integers(-3, 4, (M, K)).astype(np.float16)
+    X = rng.integers(-2, 3, (B, K)).astype(np.float16)
+    acts = rng.random((B, K)) < 0.6
+    Y, _ = O.spmspv_batch_ref(W, X, acts)
+    for b in range(B):
+        for i in range(M):
+            want = sum(float(W[i, j]) * float(X[b, j]) for j in range(K) if acts[b, j])
+            assert Y[b, i] == want
+    perm = np.array([2, 0, 1])
+    Yp, _ = O.spmspv_batch_ref(W, X[perm], acts[perm])
+    assert np.array_equal(Yp, Y[perm])                      # tokens do not interact
+    y1, _ = O.spmspv_ref(W, X[1], acts[1])
+    assert np.array_equal(Y[1], y1)                         # a batch of one is the single-vector result
+
+
+def test_batch_union_and_bytes():
+    rng = np.random.Generator(np.random.PCG64(73))
+    M, K, B = 512, 96, 4
+    W = (rng.standard_normal((M, K)) * (rng.random((M, K)) < 0.5)).astype(np.float16)
+    p = O.pack_ref(W)
+    acts = rng.random((B, K)) < 0.3
+    u = O.union_active(acts)
+    assert np.array_equal(u, acts[0] | acts[1] | acts[2] | acts[3])
+    same = np.repeat(acts[:1], B, axis=0)                   # identical tokens: matrix bytes once, vectors B times
+    assert O.active_bytes_batch(p, same) == O.active_bytes(p, acts[0]) + (B - 1) * (2 * K + 2 * M)
+    assert O.active_bytes_batch(p, acts) >= max(O.active_bytes(p, a) for a in acts)
+    assert O.active_bytes_batch(p, acts[:1]) == O.active_bytes(p, acts[0])

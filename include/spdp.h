@@ -122,6 +122,23 @@ SPDP_API spdp_status spdp_import_tiled_cbc(int64_t M, int64_t K, int pad_elems, 
 SPDP_API spdp_status spdp_spmspv(spdp_handle h, const void* x_dev, spdp_dp_rule rule, float thr,
                         const void* mask_dev, void* y_dev, spdp_ydtype ydt, void* stream);
 
+/* Small-batch decode: Y[b] = W_sp * x_b for `batch` tokens (1..SPDP_MAX_BATCH) in one pass over
+ * the packed matrix.  The paper treats one token per call and names batched DP decode as future
+ * work (Sec. 6); this entry point applies its definition token by token: token b has its own
+ * active set (the DP rule on x_b), a column tile is fetched once if ANY token keeps its column,
+ * and a token that skips a column enters the product with 0 for it.  With finite weights that is
+ * the omission of the column; a column tile that holds Inf or NaN and is fetched for another token
+ * gives NaN instead (0 * Inf).
+ *   x_dev        fp16 [batch][ldx], device, ldx >= K elements between tokens.
+ *   mask_dev     uint32 [batch][mask_stride] words, mask_stride >= ceil(K/32); SPDP_DP_MASK only.
+ *   y_dev        [batch][ldy] of ydt, ldy >= M elements between tokens; all batch*M entries are written.
+ * Asynchronous on `stream`, allocates nothing, launches one kernel; the handle's batch workspace
+ * allows one such call in flight per handle.  Results are identical from call to call. */
+#define SPDP_MAX_BATCH 8
+SPDP_API spdp_status spdp_spmspv_batch(spdp_handle h, const void* x_dev, int64_t ldx, int batch, spdp_dp_rule rule,
+                              float thr, const void* mask_dev, int64_t mask_stride, void* y_dev, int64_t ldy,
+                              spdp_ydtype ydt, void* stream);
+
 /* Same product with HOST vectors (Sec. 4.2): copies x_host (fp16 [K], ideally pinned) to a
  * staging buffer of the handle, runs spdp_spmspv, copies y back into y_host ([M] of ydt) and
  * synchronises `stream`.  mask_host is uint32[ceil(K/32)] or NULL. */

@@ -26,6 +26,7 @@ void release(spdp_matrix* h) {
     cudaFree(h->bitmap);
     cudaFree(h->values);
     cudaFree(h->workspace);
+    cudaFree(h->workspace_batch);
     cudaFree(h->status_word);
     cudaFree(h->x_stage);
     cudaFree(h->mask_stage);
@@ -65,10 +66,14 @@ spdp_status build_partition(spdp_matrix* h, int num_ctas) {
     if (P > NGT) P = static_cast<int>(NGT);
     if (P < 1) P = 1;
     cudaFree(h->workspace);     h->workspace = nullptr;
+    cudaFree(h->workspace_batch);   h->workspace_batch = nullptr;
     h->num_ctas = P;
     h->workspace_bytes = static_cast<int64_t>(P) * kTileM * sizeof(float);   // one row of split-K tree nodes per CTA
     SPDP_CUDA_TRY(cudaMalloc(&h->workspace, h->workspace_bytes));
     SPDP_CUDA_TRY(cudaMemset(h->workspace, 0, h->workspace_bytes));
+    SPDP_CUDA_TRY(cudaMalloc(&h->workspace_batch, batch_workspace_bytes(P)));
+    SPDP_CUDA_TRY(cudaMemset(h->workspace_batch, 0, batch_workspace_bytes(P)));
+    h->workspace_bytes += batch_workspace_bytes(P);
     return SPDP_OK;
 }
 
@@ -76,6 +81,8 @@ spdp_status finish_handle(spdp_matrix* h) {
     spdp_status st = build_partition(h, 0);
     if (st != SPDP_OK) return st;
     st = configure_spmspv_kernel();
+    if (st != SPDP_OK) return st;
+    st = configure_spmspv_batch_kernel();
     if (st != SPDP_OK) return st;
     SPDP_CUDA_TRY(cudaMalloc(&h->status_word, sizeof(int)));
     SPDP_CUDA_TRY(cudaMemset(h->status_word, 0, sizeof(int)));
@@ -181,6 +188,25 @@ spdp_status spdp_spmspv(spdp_handle h, const void* x_dev, spdp_dp_rule rule, flo
     if (cudaGetDevice(&dev) != cudaSuccess || dev != h->device) return SPDP_ERR_INVALID_ARG;   // wrong current device
     return launch_spmspv(h, static_cast<const __half*>(x_dev), rule, thr,
                          static_cast<const uint32_t*>(mask_dev), y_dev, ydt, static_cast<cudaStream_t>(stream));
+}
+
+spdp_status spdp_spmspv_batch(spdp_handle h, const void* x_dev, int64_t ldx, int batch, spdp_dp_rule rule, float thr,
+                              const void* mask_dev, int64_t mask_stride, void* y_dev, int64_t ldy,
+                              spdp_ydtype ydt, void* stream) {
+    if (!valid(h) || x_dev == nullptr || y_dev == nullptr) return SPDP_ERR_INVALID_ARG;
+    if (batch < 1 || batch > SPDP_MAX_BATCH || ldx < h->K || ldy < h->M) return SPDP_ERR_INVALID_ARG;
+    if (!rule_ok(rule) || (ydt != SPDP_Y_F16 && ydt != SPDP_Y_F32)) return SPDP_ERR_INVALID_ARG;
+    if (rule == SPDP_DP_MASK && (mask_dev == nullptr || mask_stride < (h->K + 31) / 32)) return SPDP_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(x_dev) & 1u) ||
+        (reinterpret_cast<uintptr_t>(y_dev) & (ydt == SPDP_Y_F32 ? 3u : 1u)) ||
+        (reinterpret_cast<uintptr_t>(mask_dev) & 3u))
+        return SPDP_ERR_INVALID_ARG;
+    if (h->pad_elems != 8) return SPDP_ERR_UNSUPPORTED_SHAPE;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev != h->device) return SPDP_ERR_INVALID_ARG;   // wrong current device
+    return launch_spmspv_batch(h, static_cast<const __half*>(x_dev), ldx, batch, rule, thr,
+                               static_cast<const uint32_t*>(mask_dev), mask_stride, y_dev, ldy, ydt,
+                               static_cast<cudaStream_t>(stream));
 }
 
 spdp_status spdp_spmspv_noalloc(const void* tileoffset_dev, const void* colinfo_dev, const void* bitmap_dev,

@@ -36,6 +36,7 @@ struct spdp_matrix {
     // contiguous ranges, one per CTA.
     int num_ctas;           // P
     float* workspace;       // device [P*256] split-K tree nodes, one row per CTA (all zero between calls)
+    float* workspace_batch; // device [P*8*256] tree nodes of the small-batch call (all zero between calls)
     int* status_word;       // device [1]
     int64_t workspace_bytes;
 
@@ -73,6 +74,13 @@ spdp_status launch_spmspv(const spdp_matrix* h, const __half* x, int rule, float
 spdp_status launch_spmspv_noalloc(const uint32_t* tileoffset, const uint32_t* colinfo, const uint64_t* bitmap,
                                   const __half* values, int64_t M, int64_t K, const __half* x, int rule,
                                   float thr, const uint32_t* mask, void* y, int ydt, cudaStream_t s);
+// spmspv_batch.cu
+int64_t batch_workspace_bytes(int num_ctas);
+spdp_status configure_spmspv_batch_kernel();   // per-device kernel attributes; idempotent
+spdp_status launch_spmspv_batch(const spdp_matrix* h, const __half* x, int64_t ldx, int batch, int rule, float thr,
+                                const uint32_t* mask, int64_t mask_stride, void* y, int64_t ldy, int ydt,
+                                cudaStream_t s);
+
 spdp_status launch_active_columns(const spdp_matrix* h, const __half* x, int rule, float thr,
                                   const uint32_t* mask, uint32_t* bits, int* count, cudaStream_t s);
 

@@ -27,7 +27,7 @@ SPDP_Y_F16, SPDP_Y_F32 = 0, 1
 
 EXPORTS = (
     "spdp_pack_tiled_cbc", "spdp_pack_tiled_cbc_ex", "spdp_import_tiled_cbc", "spdp_spmspv",
-    "spdp_spmspv_host", "spdp_spmspv_noalloc", "spdp_free", "spdp_get_info", "spdp_export", "spdp_unpack",
+    "spdp_spmspv_host", "spdp_spmspv_noalloc", "spdp_spmspv_batch", "spdp_free", "spdp_get_info", "spdp_export", "spdp_unpack",
     "spdp_active_columns", "spdp_last_device_status", "spdp_set_num_ctas", "spdp_last_cuda_error",
     "spdp_status_string",
 )
@@ -66,6 +66,7 @@ def lib():
         L.spdp_spmspv.argtypes = [vp, vp, ci, cf, vp, vp, ci, vp]
         L.spdp_spmspv_host.argtypes = [vp, vp, ci, cf, vp, vp, ci, vp]
         L.spdp_spmspv_noalloc.argtypes = [vp, vp, vp, vp, i64, i64, vp, ci, cf, vp, vp, ci, vp]
+        L.spdp_spmspv_batch.argtypes = [vp, vp, i64, ci, ci, cf, vp, i64, vp, i64, ci, vp]
         L.spdp_free.argtypes = [vp]
         L.spdp_get_info.argtypes = [vp, ctypes.POINTER(spdp_info)]
         L.spdp_export.argtypes = [vp, vp, vp, vp, vp]
@@ -187,6 +188,29 @@ def spdp_spmspv_noalloc(tileoffset, colinfo, bitmap, values, M: int, K: int, x, 
                                    ptr(values, "values"), M, K, _dev_ptr(x, "x"), rule, float(thr),
                                    _dev_ptr(mask, "mask", True), _dev_ptr(y, "y"), ydt, _stream(stream))
     _check(st, "spdp_spmspv_noalloc")
+
+
+def spdp_spmspv_batch(h: int, X, rule: int, thr: float, Y, mask=None, stream=None) -> None:
+    """Small-batch call: X fp16 CUDA [B][K] (rows may be strided), Y fp16 or fp32 CUDA [B][M], 1 <= B <= 8;
+    mask (SPDP_DP_MASK only) int32/uint32 CUDA [B][>= ceil(K/32)] words."""
+    import torch
+    if X.dim() != 2 or Y.dim() != 2 or X.shape[0] != Y.shape[0]:
+        raise ValueError("X must be [B][K] and Y [B][M]")
+    if Y.dtype not in (torch.float16, torch.float32) or X.dtype != torch.float16:
+        raise ValueError("X must be fp16 and Y fp16 or fp32")
+    if X.stride(1) != 1 or Y.stride(1) != 1 or (mask is not None and (mask.dim() != 2 or mask.stride(1) != 1)):
+        raise ValueError("the last dimension of X, Y and mask must be contiguous")
+    ydt = SPDP_Y_F32 if Y.dtype == torch.float32 else SPDP_Y_F16
+    B = int(X.shape[0])
+    ldx = int(X.stride(0)) if B > 1 else int(X.shape[1])
+    ldy = int(Y.stride(0)) if B > 1 else int(Y.shape[1])
+    mstride = 0 if mask is None else (int(mask.stride(0)) if B > 1 else int(mask.shape[1]))
+    if not X.is_cuda or not Y.is_cuda or (mask is not None and not mask.is_cuda):
+        raise ValueError("X, Y and mask must be CUDA tensors")
+    st = lib().spdp_spmspv_batch(h, X.data_ptr(), ldx, B, rule, float(thr),
+                                 None if mask is None else mask.data_ptr(), mstride, Y.data_ptr(), ldy, ydt,
+                                 _stream(stream))
+    _check(st, "spdp_spmspv_batch")
 
 
 def spdp_free(h) -> None:

@@ -1,0 +1,135 @@
+"""Small-batch decode (spdp_spmspv_batch) against the oracle's token-by-token definition."""
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+
+from oracle import spdp_oracle as O
+from paper_2607_21985_b200 import workloads as WL
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def S():
+    from paper_2607_21985_b200 import spdp
+    spdp.lib()
+    return spdp
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def check(Y, Y_ref, S_ref):
+    err = np.abs(Y.astype(np.float64) - Y_ref)
+    tol = O.tolerance(S_ref)
+    assert np.all(err <= tol), f"worst error/tolerance {np.max(err / tol):.3g}"
+
+
+def run_batch(S, h, X, rule, thr, M, ydtype=torch.float32, mask=None):
+    B = X.shape[0]
+    Y = torch.full((B, M), float("nan"), dtype=ydtype, device="cuda")
+    S.spdp_spmspv_batch(h, dev(X), rule, thr, Y, mask=None if mask is None else dev(mask))
+    torch.cuda.synchronize()
+    assert S.spdp_last_device_status(h) == 0
+    return Y.float().cpu().numpy()
+
+
+@pytest.mark.parametrize("M,K,sp,skip,seed", [
+    (256, 16, 0.5, 0.5, 1), (300, 40, 0.3, 0.25, 2), (1, 1, 0.0, 0.0, 3), (257, 17, 0.5, 0.5, 4),
+    (1024, 1024, 0.5, 0.4, 5), (768, 4400, 0.7, 0.9, 6), (2304, 528, 0.9, 0.4, 7), (256, 8192, 0.6, 0.5, 8),
+    (512, 20000, 0.5, 0.3, 9), (1000, 8200, 0.2, 0.6, 10)])
+@pytest.mark.parametrize("B", [1, 2, 3, 5, 8])
+def test_batch_matches_oracle(S, M, K, sp, skip, seed, B):
+    rw, rx = WL._rngs(seed)
+    W = WL.prune_global_magnitude(WL.normal_weights(rw, M, K), sp).astype(np.float16)
+    X = rx.standard_normal((B, K), dtype=np.float32).astype(np.float16)
+    # one threshold for the whole batch (the library takes a scalar): the first token's quantile
+    rule, thr = WL.skip_threshold(X[0], skip)
+    acts = np.stack([O.active_ref(X[b], rule, thr) for b in range(B)])
+    Y_ref, S_ref = O.spmspv_batch_ref(W, X, acts)
+    h = S.spdp_pack_tiled_cbc(dev(W))
+    try:
+        for ydtype in (torch.float32, torch.float16):
+            Y = run_batch(S, h, X, rule, thr, M, ydtype)
+            check(Y, Y_ref, S_ref)
+        Y2 = run_batch(S, h, X, rule, thr, M, torch.float16)
+        assert np.array_equal(Y, Y2)                                   # fixed summation order
+        for ctas in (1, 3, 37, 1000):                                  # other split-K layouts
+            S.spdp_set_num_ctas(h, ctas)
+            check(run_batch(S, h, X, rule, thr, M), Y_ref, S_ref)
+    finally:
+        S.spdp_free(h)
+
+
+def test_batch_with_masks_strides_and_idle_tokens(S):
+    """Per-token explicit masks, padded row strides, a token that keeps nothing and one that keeps all."""
+    rng = np.random.Generator(np.random.PCG64(31))
+    M, K, B = 700, 3000, 4
+    W = (rng.standard_normal((M, K)) * (rng.random((M, K)) < 0.4) * 0.05).astype(np.float16)
+    X = rng.standard_normal((B, K)).astype(np.float16)
+    acts = rng.random((B, K)) < 0.35
+    acts[1] = False
+    acts[2] = True
+    words = np.stack([O.active_to_words(a) for a in acts])
+    Y_ref, S_ref = O.spmspv_batch_ref(W, X, acts)
+    h = S.spdp_pack_tiled_cbc(dev(W))
+    try:
+        Xd = torch.zeros((B, K + 24), dtype=torch.float16, device="cuda")
+        Xd[:, :K] = dev(X)
+        Yd = torch.full((B, M + 5), float("nan"), dtype=torch.float32, device="cuda")
+        md = torch.zeros((B, words.shape[1] + 3), dtype=torch.int32, device="cuda")
+        md[:, :words.shape[1]] = dev(words.view(np.int32))
+        S.spdp_spmspv_batch(h, Xd[:, :K], O.DP_MASK, 0.0, Yd[:, :M], mask=md[:, :words.shape[1]])
+        torch.cuda.synchronize()
+        out = Yd.cpu().numpy()
+        check(out[:, :M], Y_ref, S_ref)
+        assert np.all(out[1, :M] == 0.0)                               # nothing kept: zeros, still written
+        assert np.all(np.isnan(out[:, M:]))                            # nothing written beyond M
+        # odd row stride: the slices of x are no longer 16-byte aligned
+        Xo = torch.zeros((B, K + 3), dtype=torch.float16, device="cuda")
+        Xo[:, :K] = dev(X)
+        Yo = torch.empty((B, M), dtype=torch.float32, device="cuda")
+        S.spdp_spmspv_batch(h, Xo[:, :K], O.DP_MASK, 0.0, Yo, mask=md[:, :words.shape[1]])
+        torch.cuda.synchronize()
+        check(Yo.cpu().numpy(), Y_ref, S_ref)
+    finally:
+        S.spdp_free(h)
+
+
+def test_batch_exact_on_integers_and_agrees_with_single_vector_calls(S):
+    rng = np.random.Generator(np.random.PCG64(32))
+    M, K, B = 900, 1200, 8
+    W = rng.integers(-8, 9, (M, K)).astype(np.float16)
+    W[rng.random((M, K)) < 0.6] = 0
+    X = rng.integers(-4, 5, (B, K)).astype(np.float16)
+    acts = np.stack([O.active_ref(X[b], O.DP_ABS_GT, 1.0) for b in range(B)])
+    Y_ref, _ = O.spmspv_batch_ref(W, X, acts)
+    h = S.spdp_pack_tiled_cbc(dev(W))
+    try:
+        Y = run_batch(S, h, X, O.DP_ABS_GT, 1.0, M)
+        assert np.array_equal(Y, Y_ref)                                # every partial sum is exact
+        for b in range(B):
+            y1 = torch.empty(M, dtype=torch.float32, device="cuda")
+            S.spdp_spmspv(h, dev(X[b]), O.DP_ABS_GT, 1.0, y1)
+            torch.cuda.synchronize()
+            assert np.array_equal(y1.cpu().numpy(), Y[b])
+    finally:
+        S.spdp_free(h)
+
+
+def test_batch_rejects_bad_arguments(S):
+    W = torch.zeros((256, 32), dtype=torch.float16, device="cuda")
+    h = S.spdp_pack_tiled_cbc(W)
+    try:
+        Y9 = torch.zeros((9, 256), dtype=torch.float32, device="cuda")
+        X9 = torch.zeros((9, 32), dtype=torch.float16, device="cuda")
+        with pytest.raises(S.SpdpError, match="INVALID_ARG"):
+            S.spdp_spmspv_batch(h, X9, 0, 0.0, Y9)                     # more than 8 tokens
+        with pytest.raises(S.SpdpError, match="INVALID_ARG"):
+            S.spdp_spmspv_batch(h, X9[:2], 2, 0.0, Y9[:2])             # mask rule without masks
+        with pytest.raises(S.SpdpError, match="INVALID_ARG"):
+            S.spdp_spmspv_batch(h, X9[:1], 0, 0.0, Y9[:1, :100].contiguous())   # fewer than M outputs per token
+    finally:
+        S.spdp_free(h)

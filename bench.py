@@ -210,6 +210,83 @@ def run_reference(args):
     }))
 
 
+def run_batch(args):
+    """--batch B: the small-batch entry point (spdp_spmspv_batch) on the same layer, B tokens with
+    independent activations and the same skip fraction.  A side measurement, not the headline."""
+    import torch
+    from paper_2607_21985_b200 import spdp
+    from paper_2607_21985_b200 import workloads as WL
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    spdp.lib()
+    w = make_workload(args.workload)
+    B = args.batch
+    rng = np.random.Generator(np.random.PCG64(np.random.SeedSequence(9000 + B)))
+    X = np.concatenate([w.x[None, :], rng.standard_normal((B - 1, w.K), dtype=np.float32).astype(np.float16)])
+    l2 = torch.cuda.get_device_properties(0).L2_cache_size
+    Wd = torch.from_numpy(w.W).cuda()
+    h0 = spdp.spdp_pack_tiled_cbc(Wd)
+    info = spdp.spdp_get_info(h0)
+    Xd = torch.from_numpy(X).cuda()
+    union = np.zeros((w.K + 31) // 32, dtype=np.uint32)
+    per_token = []
+    for b in range(B):
+        words = torch.zeros((w.K + 31) // 32, dtype=torch.int32, device="cuda")
+        spdp.spdp_active_columns(h0, Xd[b], w.rule, w.thr, words)
+        torch.cuda.synchronize()
+        wb = words.cpu().numpy().view(np.uint32)
+        per_token.append(int(np.unpackbits(wb.view(np.uint8)).sum()))
+        union |= wb
+    n_union = int(np.unpackbits(union.view(np.uint8)).sum())
+    B_active = active_bytes(spdp.spdp_export(h0)["colinfo"], union, w.M, w.K, 2) + (B - 1) * (2 * w.K + 2 * w.M)
+    copies = args.copies or max(2, int(np.ceil(2 * l2 / B_active)) + 1)
+    handles = [h0] + [spdp.spdp_pack_tiled_cbc(Wd) for _ in range(copies - 1)]
+    Xs = [Xd.clone() for _ in range(copies)]
+    Ys = [torch.empty((B, w.M), dtype=torch.float16, device="cuda") for _ in range(copies)]
+    ys1 = [torch.empty(w.M, dtype=torch.float16, device="cuda") for _ in range(copies)]
+
+    def timed(fn, steps):
+        for i in range(args.warmup):
+            fn(i)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(steps):
+            fn(i)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / steps * 1e3
+
+    us_batch = timed(lambda i: spdp.spdp_spmspv_batch(handles[i % copies], Xs[i % copies], w.rule, w.thr, Ys[i % copies]),
+                     args.steps)
+
+    def one_by_one(i):
+        k = i % copies
+        for b in range(B):
+            spdp.spdp_spmspv(handles[k], Xs[k][b], w.rule, w.thr, ys1[k])
+    us_single = timed(one_by_one, max(20, args.steps // B))
+    Ws = [Wd, Wd.clone()]
+    XT = Xd.t().contiguous()
+    us_dense = timed(lambda i: torch.mm(Ws[i % 2], XT), 50)
+    peak, peak_kind = measured_peak()
+    achieved = B_active / (us_batch * 1e-6) / 1e9
+    print(json.dumps({
+        "metric": "spmspv_batch_effective_hbm_gbs", "value": achieved, "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": us_batch * 1e-3, "us_per_call": us_batch, "us_per_token": us_batch / B,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "batch": B, "active_columns_per_token": per_token, "active_columns_union": n_union,
+                   "active_bytes_per_call": int(B_active), "packed_bytes": int(info.packed_bytes), "copies": copies,
+                   "l2": "inputs larger than L2: rotating packed copies"},
+        "gpu_launches": args.steps,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "peak_kind": f"of {peak_kind}", "traffic": None, "kernel": "spmspv_batch_kernel",
+                     "algorithmic_bytes": int(B_active)},
+        "context": {"same_tokens_one_call_each_us": us_single, "dense_fp16_gemm_us": us_dense,
+                    "dense_bytes": int(2 * w.M * w.K)},
+    }))
+    for h in handles:
+        spdp.spdp_free(h)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -222,11 +299,15 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-context", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay timing")
+    ap.add_argument("--batch", type=int, default=1, help="2..8: time the small-batch entry point instead (1 GPU)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.batch > 1:
+        run_batch(args)
         return
 
     import torch

@@ -29,7 +29,8 @@ constexpr int kWarps = 16;
 constexpr int kThreads = kWarps * 32;
 constexpr int kDepth = 2;                    // K-blocks a warp keeps in flight
 constexpr int kBlockTiles = 8;               // active column tiles per K-block (the K of the instruction)
-constexpr int kSlotBytes = 2 * kTileM + 32;
+constexpr int kSlotBytes = 2 * kTileM + 16;   // 16 bytes more than a full column tile: the four tiles whose values the
+                                             // lanes of one load read (every second slot) start 8 banks apart
 constexpr int kStageBytes = kBlockTiles * kSlotBytes;
 constexpr int kChunkCols = 2048;             // columns listed per batch
 constexpr int kChunkGT = kChunkCols / kTileK;
@@ -92,11 +93,45 @@ __device__ __forceinline__ unsigned lds_u16(uint32_t addr) {
     asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(addr));
     return v;
 }
-// The fp16 value of the bitmap position `bit` of word W (whose first value sits at `first`), or 0.
-__device__ __forceinline__ unsigned pick(unsigned W, uint32_t first, unsigned below, unsigned bit) {
-    unsigned v = 0;
-    if (W & bit) v = lds_u16(first + 2u * __popc(W & below));
-    return v;
+// Rebuilds this lane's part of two fragments from one 32-bit bitmap word of two column tiles (Sec. 4.2.1):
+// WA / WB are the word of tile A / B, FA / FB the shared-memory address of the word's first value,
+// bit k = my row inside the k-th 8-row slice of the word, below k = the bits before it.  A set bit
+// takes the value at rank = set bits before it; a clear bit gives 0.  Output k packs (tile A, tile B)
+// for bit k, which is what the tensor-core fragment wants (two adjacent K indices per register).
+// (Ranking 2 or 4 adjacent rows with one popcount needs fewer instructions but spreads the 32
+// simultaneous loads over more banks; measured 134 and 140 us against 125 us on the largest layer.)
+#define SPDP_PICK(V, W, F, BELOW, BIT)                      \
+    " and.b32 t, " W ", " BELOW ";\n"                      \
+    " popc.b32 t, t;\n"                                    \
+    " shl.b32 t, t, 1;\n"                                  \
+    " add.u32 t, t, " F ";\n"                              \
+    " and.b32 s, " W ", " BIT ";\n"                        \
+    " setp.ne.u32 p, s, 0;\n"                              \
+    " mov.b16 " V ", 0;\n"                                 \
+    " @p ld.shared.u16 " V ", [t];\n"
+__device__ __forceinline__ void rebuild_word(unsigned (&a)[4], unsigned WA, unsigned FA, unsigned WB, unsigned FB,
+                                             const unsigned (&below)[4], const unsigned (&bit)[4]) {
+    asm volatile(
+        "{\n"
+        " .reg .pred p;\n"
+        " .reg .b16 v0, v1, v2, v3, u0, u1, u2, u3;\n"
+        " .reg .b32 t, s;\n"
+        SPDP_PICK("v0", "%4", "%5", "%8", "%12")
+        SPDP_PICK("u0", "%6", "%7", "%8", "%12")
+        SPDP_PICK("v1", "%4", "%5", "%9", "%13")
+        SPDP_PICK("u1", "%6", "%7", "%9", "%13")
+        SPDP_PICK("v2", "%4", "%5", "%10", "%14")
+        SPDP_PICK("u2", "%6", "%7", "%10", "%14")
+        SPDP_PICK("v3", "%4", "%5", "%11", "%15")
+        SPDP_PICK("u3", "%6", "%7", "%11", "%15")
+        " mov.b32 %0, {v0, u0};\n"
+        " mov.b32 %1, {v1, u1};\n"
+        " mov.b32 %2, {v2, u2};\n"
+        " mov.b32 %3, {v3, u3};\n"
+        "}"
+        : "=r"(a[0]), "=r"(a[1]), "=r"(a[2]), "=r"(a[3])
+        : "r"(WA), "r"(FA), "r"(WB), "r"(FB), "r"(below[0]), "r"(below[1]), "r"(below[2]), "r"(below[3]),
+          "r"(bit[0]), "r"(bit[1]), "r"(bit[2]), "r"(bit[3]));
 }
 // D += A (16 rows x 8 column tiles, fp16) * B (8 column tiles x 8 tokens, fp16), fp32 accumulate.
 __device__ __forceinline__ void mma_16x8x8(float (&c)[4], unsigned a01, unsigned a23, unsigned b01) {
@@ -315,14 +350,13 @@ spmspv_batch_kernel(const Params p) {
                 const uint4 wB = lds_v4<32>(tA + 16 * h), fB = lds_v4<kVoFromBm + 32>(tA + 16 * h);
                 const unsigned WA[4] = {wA.x, wA.y, wA.z, wA.w}, FA[4] = {fA.x, fA.y, fA.z, fA.w};
                 const unsigned WB[4] = {wB.x, wB.y, wB.z, wB.w}, FB[4] = {fB.x, fB.y, fB.z, fB.w};
+                unsigned a[4][4];                                                    // [word][bit gid + 8k]: (tile tA, tile tB)
+#pragma unroll
+                for (int w = 0; w < 4; ++w) rebuild_word(a[w], WA[w], FA[w], WB[w], FB[w], belowk, bitk);
 #pragma unroll
                 for (int w = 0; w < 4; ++w) {                                        // rows 32 * (4h + w) ..
-                    unsigned a[4];
-#pragma unroll
-                    for (int k = 0; k < 4; ++k)                                      // bit gid + 8k: (tile tA, tile tB)
-                        a[k] = pick(WA[w], FA[w], belowk[k], bitk[k]) | (pick(WB[w], FB[w], belowk[k], bitk[k]) << 16);
-                    mma_16x8x8(acc[2 * (4 * h + w)], a[0], a[1], b01);
-                    mma_16x8x8(acc[2 * (4 * h + w) + 1], a[2], a[3], b01);
+                    mma_16x8x8(acc[2 * (4 * h + w)], a[w][0], a[w][1], b01);
+                    mma_16x8x8(acc[2 * (4 * h + w) + 1], a[w][2], a[w][3], b01);
                 }
             }
             __syncwarp();                  // everyone is done with this ring position

@@ -60,3 +60,26 @@ def test_full_size_layer(S, c_oracle, name):
             assert np.all(err <= tol), f"{name}: worst error/tolerance {np.nanmax(err / tol):.3g}"
     finally:
         S.spdp_free(h)
+
+
+@pytest.mark.parametrize("name,B", [("c4", 8), ("c1", 5), ("c3", 8)])
+def test_full_size_small_batch(S, c_oracle, name, B):
+    """The small-batch entry point at full size, default CTA count, fp16 outputs: every token against
+    the C oracle's single-vector result for that token."""
+    w = CASES[name]()
+    rng = np.random.Generator(np.random.PCG64(np.random.SeedSequence(500 + B)))
+    X = np.concatenate([w.x[None, :], rng.standard_normal((B - 1, w.K), dtype=np.float32).astype(np.float16)])
+    h = S.spdp_pack_tiled_cbc(torch.from_numpy(w.W).cuda())
+    try:
+        Y = torch.full((B, w.M), float("nan"), dtype=torch.float16, device="cuda")
+        S.spdp_spmspv_batch(h, torch.from_numpy(X).cuda(), w.rule, w.thr, Y)
+        torch.cuda.synchronize()
+        out = Y.cpu().numpy().astype(np.float64)
+        for b in range(B):
+            a = c_oracle.active(X[b], w.rule, w.thr)
+            y_ref, S_ref, _ = c_oracle.spmspv(w.W, X[b], a)
+            err = np.abs(out[b] - y_ref)
+            tol = O.tolerance(S_ref)
+            assert np.all(err <= tol), f"{name} token {b}: worst error/tolerance {np.nanmax(err / tol):.3g}"
+    finally:
+        S.spdp_free(h)

@@ -132,8 +132,9 @@ SPDP_API spdp_status spdp_spmspv(spdp_handle h, const void* x_dev, spdp_dp_rule 
  *   x_dev        fp16 [batch][ldx], device, ldx >= K elements between tokens.
  *   mask_dev     uint32 [batch][mask_stride] words, mask_stride >= ceil(K/32); SPDP_DP_MASK only.
  *   y_dev        [batch][ldy] of ydt, ldy >= M elements between tokens; all batch*M entries are written.
- * Asynchronous on `stream`, allocates nothing, launches one kernel; the handle's batch workspace
- * allows one such call in flight per handle.  Results are identical from call to call. */
+ * Asynchronous on `stream`, allocates nothing; launches one kernel for 3 or more tokens and one
+ * single-vector kernel per token below that (which is faster there).  The handle's workspaces allow
+ * one such call in flight per handle.  Results are identical from call to call. */
 #define SPDP_MAX_BATCH 8
 SPDP_API spdp_status spdp_spmspv_batch(spdp_handle h, const void* x_dev, int64_t ldx, int batch, spdp_dp_rule rule,
                               float thr, const void* mask_dev, int64_t mask_stride, void* y_dev, int64_t ldy,

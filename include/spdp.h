@@ -128,7 +128,9 @@ SPDP_API spdp_status spdp_spmspv(spdp_handle h, const void* x_dev, spdp_dp_rule 
  * active set (the DP rule on x_b), a column tile is fetched once if ANY token keeps its column,
  * and a token that skips a column enters the product with 0 for it.  With finite weights that is
  * the omission of the column; a column tile that holds Inf or NaN and is fetched for another token
- * gives NaN instead (0 * Inf).
+ * gives NaN instead (0 * Inf).  Likewise a NaN or Inf activation of a kept column reaches, through the
+ * zeros of the fetched tiles, every row (0 * NaN), as in a dense product; the single-vector call
+ * multiplies stored nonzeros only.
  *   x_dev        fp16 [batch][ldx], device, ldx >= K elements between tokens.
  *   mask_dev     uint32 [batch][mask_stride] words, mask_stride >= ceil(K/32); SPDP_DP_MASK only.
  *   y_dev        [batch][ldy] of ydt, ldy >= M elements between tokens; all batch*M entries are written.

@@ -83,7 +83,7 @@ struct __align__(128) Smem {
 };
 static_assert(sizeof(Smem) <= 227 * 1024, "shared memory of one CTA");
 static_assert(offsetof(Smem, rec) % 16 == 0 && offsetof(Smem, xact) % 16 == 0 && offsetof(Smem, tab) % 16 == 0, "aligned tables");
-static_assert(kChunkCols / 8 <= kThreads, "one list pass");
+static_assert(kChunkCols / 4 <= kThreads, "one list pass, 4 columns per thread");
 static_assert(kRecPad <= kThreads, "one thread per trailing null record");
 static_assert(sizeof(float) * kWarps * kBT * kRedPlane + 4 * (kChunkCols + kChunkGT) + 2 * kBT * kChunkCols <=
                   size_t(kWarps) * kDepth * kStageBytes, "staging must fit in the ring behind red");
@@ -133,6 +133,20 @@ __device__ __forceinline__ void rebuild_word(unsigned (&a)[4], unsigned WA, unsi
         : "r"(WA), "r"(FA), "r"(WB), "r"(FB), "r"(below[0]), "r"(below[1]), "r"(below[2]), "r"(below[3]),
           "r"(bit[0]), "r"(bit[1]), "r"(bit[2]), "r"(bit[3]));
 }
+// The DP test of Sec. 4.2 step (3) on a pair of fp16 activations: 0xFFFF in each half whose column is
+// kept, i.e. NOT(|x| <= thr).  thr2 holds, twice, the largest fp16 value that does not exceed thr:
+// for an fp16 x that is the same test as the fp32 comparison, and "greater than or unordered" keeps
+// NaN activations and makes a NaN threshold keep everything, as the fp32 form does.
+__device__ __forceinline__ unsigned abs_gt_keep(unsigned x2, unsigned thr2) {
+    unsigned r;
+    asm("{\n .reg .b32 a;\n and.b32 a, %1, 0x7FFF7FFF;\n set.gtu.u32.f16x2 %0, a, %2;\n}" : "=r"(r) : "r"(x2), "r"(thr2));
+    return r;
+}
+__device__ __forceinline__ unsigned threshold_pair(float thr) {
+    unsigned short h;
+    asm("cvt.rm.f16.f32 %0, %1;" : "=h"(h) : "f"(thr));
+    return static_cast<unsigned>(h) * 0x00010001u;
+}
 // D += A (16 rows x 8 column tiles, fp16) * B (8 column tiles x 8 tokens, fp16), fp32 accumulate.
 __device__ __forceinline__ void mma_16x8x8(float (&c)[4], unsigned a01, unsigned a23, unsigned b01) {
     asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%0,%1,%2,%3};"
@@ -166,6 +180,8 @@ spmspv_batch_kernel(const Params p) {
     const uint32_t x_addr = smem_u32(&sm.xact[0][0]);
     const unsigned char* const val_src = reinterpret_cast<const unsigned char*>(p.values) + 16 * lane7;
     const unsigned char* const bm_src = reinterpret_cast<const unsigned char*>(p.bitmap) + 4 * lane7;
+
+    const unsigned thr2 = threshold_pair(p.thr);
 
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     bool waited_for_stream = false;
@@ -217,38 +233,36 @@ spmspv_batch_kernel(const Params p) {
         __syncthreads();
 
         // ---- (2) active list of the union of the tokens' active sets ----
-        // A thread takes 8 consecutive columns: one 8-bit mask per token, their union decides which
-        // column tiles get a record; a token's activations are zeroed where it skips the column.
-        const int v0 = t * 8;
+        // A thread takes 4 consecutive columns: per token the DP test on two fp16 pairs gives a keep
+        // mask (0xFFFF per kept half), which zeroes the activations the token skips; the union of the
+        // tokens' bits decides which column tiles get a record.
+        const int v0 = t * 4;
         unsigned m = 0;
-        unsigned xs[kBT][4];                 // my 8 columns' activations per token (fp16 pairs), skipped ones zeroed
+        unsigned xs[kBT][2];                 // my 4 columns' activations per token (fp16 pairs), skipped ones zeroed
+        {
+            const int lim = n - v0;                                         // positions of mine that hold a column
+            const unsigned valid0 = lim >= 2 ? 0xFFFFFFFFu : (lim == 1 ? 0x0000FFFFu : 0u);
+            const unsigned valid1 = lim >= 4 ? 0xFFFFFFFFu : (lim == 3 ? 0x0000FFFFu : 0u);
 #pragma unroll
-        for (int b = 0; b < kBT; ++b) {
-            xs[b][0] = xs[b][1] = xs[b][2] = xs[b][3] = 0u;
-            if (b < p.batch && v0 < n) {
-                const uint4 xv = *reinterpret_cast<const uint4*>(&sm.stage.x[b][v0]);
-                unsigned xw[4] = {xv.x, xv.y, xv.z, xv.w};
-                unsigned mb = 0xFFu;
-                if (p.rule == SPDP_DP_ABS_GT) {
-                    mb = 0;
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const float lo = __half2float(__ushort_as_half(static_cast<unsigned short>(xw[i] & 0xFFFFu)));
-                        const float hi = __half2float(__ushort_as_half(static_cast<unsigned short>(xw[i] >> 16)));
-                        mb |= (!(fabsf(lo) <= p.thr) ? 1u : 0u) << (2 * i);
-                        mb |= (!(fabsf(hi) <= p.thr) ? 1u : 0u) << (2 * i + 1);
+            for (int b = 0; b < kBT; ++b) {
+                xs[b][0] = xs[b][1] = 0u;
+                if (b < p.batch && lim > 0) {
+                    const uint2 xv = *reinterpret_cast<const uint2*>(&sm.stage.x[b][v0]);
+                    unsigned k0 = 0xFFFFFFFFu, k1 = 0xFFFFFFFFu;
+                    if (p.rule == SPDP_DP_ABS_GT) {
+                        k0 = abs_gt_keep(xv.x, thr2);
+                        k1 = abs_gt_keep(xv.y, thr2);
+                    } else if (p.rule == SPDP_DP_MASK) {
+                        const int j = j0 + v0;                              // a multiple of 4
+                        const unsigned bits = __ldg(p.mask + b * p.mask_stride + (j >> 5)) >> (j & 31);
+                        k0 = ((bits & 1u) ? 0x0000FFFFu : 0u) | ((bits & 2u) ? 0xFFFF0000u : 0u);
+                        k1 = ((bits & 4u) ? 0x0000FFFFu : 0u) | ((bits & 8u) ? 0xFFFF0000u : 0u);
                     }
-                } else if (p.rule == SPDP_DP_MASK) {
-                    const int j = j0 + v0;                                  // a multiple of 8
-                    mb = (__ldg(p.mask + b * p.mask_stride + (j >> 5)) >> (j & 31)) & 0xFFu;
-                }
-                const int lim = n - v0;
-                mb &= (lim >= 8) ? 0xFFu : ((1u << lim) - 1u);
-                m |= mb;
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const unsigned keep = (((mb >> (2 * i)) & 1u) ? 0x0000FFFFu : 0u) | (((mb >> (2 * i + 1)) & 1u) ? 0xFFFF0000u : 0u);
-                    xs[b][i] = xw[i] & keep;
+                    k0 &= valid0;
+                    k1 &= valid1;
+                    xs[b][0] = xv.x & k0;
+                    xs[b][1] = xv.y & k1;
+                    m |= (k0 & 1u) | ((k0 >> 30) & 2u) | ((k1 & 1u) << 2) | ((k1 >> 28) & 8u);
                 }
             }
         }
@@ -270,11 +284,10 @@ spmspv_batch_kernel(const Params p) {
                 const unsigned slot0 = gA * kTileK + v0;                    // column slot of position v0
                 int item = static_cast<int>(base + inc - cnt);
                 const unsigned to = sm.stage.tileoff[v0 >> 4];
-                const uint4 c0v = *reinterpret_cast<const uint4*>(&sm.stage.colinfo[v0]);
-                const uint4 c1v = *reinterpret_cast<const uint4*>(&sm.stage.colinfo[v0 + 4]);
-                const unsigned ci[8] = {c0v.x, c0v.y, c0v.z, c0v.w, c1v.x, c1v.y, c1v.z, c1v.w};
+                const uint4 cv = *reinterpret_cast<const uint4*>(&sm.stage.colinfo[v0]);
+                const unsigned ci[4] = {cv.x, cv.y, cv.z, cv.w};
 #pragma unroll
-                for (int k = 0; k < 8; ++k) {
+                for (int k = 0; k < 4; ++k) {
                     if ((m >> k) & 1u) {
                         sm.rec[item] = make_uint2(to + (ci[k] >> 16), ((slot0 + k) << 6) | (((ci[k] & 0xFFFFu) + 7u) >> 3));
                         uint4 xr;
@@ -370,8 +383,10 @@ spmspv_batch_kernel(const Params p) {
         if (done) {
             const int q0 = range_owner(ngt_all, nctas, static_cast<unsigned>(r) * p.C);
             const int nseg = range_owner(ngt_all, nctas, static_cast<unsigned>(r + 1) * p.C - 1u) - q0 + 1;
+            const int tok = t >> 6, rr = t & 63;                // my output in every 64-row chunk
+            float part[4];
 #pragma unroll
-            for (int ch = 0; ch < 4; ++ch) {                    // 64 rows at a time
+            for (int ch = 0; ch < 4; ++ch) {                    // 64 rows at a time through the idle ring
 #pragma unroll
                 for (int rbl = 0; rbl < 4; ++rbl) {
                     float (&c)[4] = acc[4 * ch + rbl];
@@ -382,19 +397,43 @@ spmspv_batch_kernel(const Params p) {
                     c[0] = c[1] = c[2] = c[3] = 0.f;
                 }
                 __syncthreads();
-                {
-                    const int tok = t >> 6, rr = t & 63;
-                    float part = 0.f;
+                float sum = 0.f;
 #pragma unroll
-                    for (int w = 0; w < kWarps; ++w) part += sm.red[w][tok][rr];
-                    const int64_t row = static_cast<int64_t>(r) * kTileM + 64 * ch + rr;
-                    if (tok < p.batch && row < p.M) {
-                        unsigned* nodes = reinterpret_cast<unsigned*>(p.workspace) + tok * kTileM + 64 * ch + rr;
-                        if (tree_combine(part, nodes, kNodeStride, q0, nseg, static_cast<int>(blockIdx.x) - q0))
-                            store_y(p.y, p.ydt, tok * p.ldy + row, part);
+                for (int w = 0; w < kWarps; ++w) sum += sm.red[w][tok][rr];
+                part[ch] = sum;
+                __syncthreads();
+            }
+            // The four outputs walk the same tree (same segments); their exchanges at a level are
+            // issued together, so the walk costs one round trip per level, not four.
+            if (tok < p.batch) {
+                unsigned* nodes = reinterpret_cast<unsigned*>(p.workspace) + tok * kTileM + rr;
+                const int64_t row0 = static_cast<int64_t>(r) * kTileM + rr;
+                bool alive[4];
+#pragma unroll
+                for (int ch = 0; ch < 4; ++ch) alive[ch] = row0 + 64 * ch < p.M;
+                int idx = static_cast<int>(blockIdx.x) - q0;
+                for (int nn = nseg, level = 0; nn > 1; nn = (nn + 1) >> 1, ++level, idx >>= 1) {
+                    const int right = idx | 1;
+                    if (right >= nn) continue;                  // no neighbour at this level
+                    unsigned* node = nodes + static_cast<int64_t>(q0 + (right << level)) * kNodeStride;
+                    unsigned old[4];
+#pragma unroll
+                    for (int ch = 0; ch < 4; ++ch)
+                        if (alive[ch]) old[ch] = atomicExch(node + 64 * ch, canonical_bits(part[ch]) ^ kNodeKey);
+#pragma unroll
+                    for (int ch = 0; ch < 4; ++ch) {
+                        if (!alive[ch]) continue;
+                        if (old[ch] == 0u) {
+                            alive[ch] = false;                  // first at the node: the neighbour carries the sum on
+                        } else {
+                            node[64 * ch] = 0u;                 // second: empty the node for the next call
+                            part[ch] += __uint_as_float(old[ch] ^ kNodeKey);
+                        }
                     }
                 }
-                __syncthreads();
+#pragma unroll
+                for (int ch = 0; ch < 4; ++ch)
+                    if (alive[ch]) store_y(p.y, p.ydt, tok * p.ldy + row0 + 64 * ch, part[ch]);
             }
         }
     }

@@ -133,3 +133,34 @@ def test_batch_rejects_bad_arguments(S):
             S.spdp_spmspv_batch(h, X9[:1], 0, 0.0, Y9[:1, :100].contiguous())   # fewer than M outputs per token
     finally:
         S.spdp_free(h)
+
+
+@pytest.mark.parametrize("thr", [0.5, 0.50006103515625, 0.3, 0.0, -0.0, -1.0, 1e-10, 70000.0, float("inf"), float("nan"),
+                                 6.1e-5, 5.96e-8])
+def test_batch_active_sets_on_threshold_edges(S, thr):
+    """W = identity, so y shows each token's active set exactly: values at, just below and just above the
+    threshold (in fp16 steps), zeros of both signs, subnormals and the largest finite values.  (Activations
+    are kept finite: the tensor-core product multiplies the zeros of a fetched tile with x, so a NaN or Inf
+    activation would mark every row of its K-block, which is the dense reading of the definition.)"""
+    K = 64
+    W = np.eye(K, dtype=np.float16)
+    base = np.float16(thr) if np.isfinite(thr) and abs(thr) < 65504 else np.float16(1.0)
+    around = [base, np.nextafter(base, np.float16(np.inf)), np.nextafter(base, np.float16(-np.inf)),
+              -base, np.float16(0.0), np.float16(-0.0), np.float16(6e-8), np.float16(-6e-8), np.float16(6.1e-5),
+              np.float16(65504), np.float16(-65504),
+              np.float16(0.25), np.float16(0.5), np.float16(0.75)]
+    rng = np.random.Generator(np.random.PCG64(77))
+    X = np.zeros((3, K), dtype=np.float16)
+    for b in range(3):
+        vals = np.array(around, dtype=np.float16)
+        X[b, :len(vals)] = rng.permutation(vals)
+        X[b, len(vals):] = rng.standard_normal(K - len(vals)).astype(np.float16)
+    acts = np.stack([O.active_ref(X[b], O.DP_ABS_GT, thr) for b in range(3)])
+    h = S.spdp_pack_tiled_cbc(dev(W))
+    try:
+        Y = run_batch(S, h, X, O.DP_ABS_GT, thr, K)
+        for b in range(3):
+            want = np.where(acts[b], X[b].astype(np.float32), np.float32(0.0))
+            assert np.array_equal(Y[b], want), (thr, b)
+    finally:
+        S.spdp_free(h)

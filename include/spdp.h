@@ -144,7 +144,10 @@ SPDP_API spdp_status spdp_spmspv_batch(spdp_handle h, const void* x_dev, int64_t
 
 /* Same product with HOST vectors (Sec. 4.2): copies x_host (fp16 [K], ideally pinned) to a
  * staging buffer of the handle, runs spdp_spmspv, copies y back into y_host ([M] of ydt) and
- * synchronises `stream`.  mask_host is uint32[ceil(K/32)] or NULL. */
+ * synchronises `stream`.  mask_host is uint32[ceil(K/32)] or NULL.  When the same pinned buffers and
+ * arguments come twice in a row, the three operations are recorded once as a CUDA graph (on a private
+ * stream of the handle) and later calls with those arguments replay it with one launch; pageable
+ * buffers, changing arguments or a stream that is being captured take the plain path. */
 SPDP_API spdp_status spdp_spmspv_host(spdp_handle h, const void* x_host, spdp_dp_rule rule, float thr,
                              const void* mask_host, void* y_host, spdp_ydtype ydt, void* stream);
 

@@ -44,6 +44,21 @@ struct spdp_matrix {
     __half* x_stage;        // device [K]
     uint32_t* mask_stage;   // device [ceil(K/32)]
     void* y_stage;          // device [M] fp32-sized
+
+    // spdp_spmspv_host with the same pinned buffers and arguments as the call before: the three
+    // operations (copy in, kernel, copy out) are kept as one instantiated graph and replayed.
+    struct HostCallKey {
+        const void* x;
+        const void* mask;
+        void* y;
+        int rule, ydt, num_ctas;
+        float thr;
+    };
+    HostCallKey host_last;          // arguments of the previous host-vector call
+    bool host_last_valid;
+    HostCallKey host_graph_key;     // arguments the graph below was recorded with
+    cudaGraphExec_t host_graph;     // null: none
+    cudaStream_t capture_stream;    // private stream used only to record that graph
 };
 
 namespace spdp {

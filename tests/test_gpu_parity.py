@@ -323,6 +323,37 @@ def test_host_vector_entry_point(S):
         S.spdp_free(h)
 
 
+def test_host_vector_entry_point_repeated_calls(S):
+    """The same pinned buffers call after call (the library may replay a recorded graph): new contents
+    of x must give new results, and a different CTA count, other buffers or pageable memory still work."""
+    rng = np.random.Generator(np.random.PCG64(91))
+    M, K = 1300, 2100
+    W = (rng.standard_normal((M, K)) * (rng.random((M, K)) < 0.5) * 0.05).astype(np.float16)
+    h = S.spdp_pack_tiled_cbc(dev(W))
+    try:
+        xh = torch.zeros(K, dtype=torch.float16).pin_memory()
+        yh = torch.zeros(M, dtype=torch.float32).pin_memory()
+        for step in range(6):
+            x = rng.standard_normal(K).astype(np.float16)
+            xh.copy_(torch.from_numpy(x))
+            yh.fill_(float("nan"))
+            if step == 4:
+                S.spdp_set_num_ctas(h, 37)
+            S.spdp_spmspv_host(h, xh, O.DP_ABS_GT, 0.4, yh)
+            a = O.active_ref(x, O.DP_ABS_GT, 0.4)
+            y_ref, S_ref = O.spmspv_ref(W, x, a)
+            check_y(yh.numpy().astype(np.float64), y_ref, S_ref)
+        y2 = torch.zeros(M, dtype=torch.float16).pin_memory()          # another output buffer and dtype
+        S.spdp_spmspv_host(h, xh, O.DP_ABS_GT, 0.4, y2)
+        check_y(y2.numpy().astype(np.float64), y_ref, S_ref)
+        yn = np.full(M, np.nan, np.float32)                            # pageable memory
+        for _ in range(3):
+            S.spdp_spmspv_host(h, x, O.DP_ABS_GT, 0.4, yn)
+            check_y(yn.astype(np.float64), y_ref, S_ref)
+    finally:
+        S.spdp_free(h)
+
+
 @pytest.mark.parametrize("make", [lambda: WL.config1(1024, 1024), lambda: WL.config2(1536, 1024),
                                   lambda: WL.config3(1024, 2752), lambda: WL.config4(3584, 1024),
                                   lambda: WL.config5(0, 0, 1024, 1024), lambda: WL.config5(3, 3, 1024, 1024)])

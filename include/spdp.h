@@ -42,7 +42,7 @@ typedef enum {
     SPDP_ERR_ALLOC = -3,             /* device or host allocation failed                        */
     SPDP_ERR_CUDA = -4,              /* a CUDA runtime call failed (see spdp_last_cuda_error)    */
     SPDP_ERR_OVERFLOW = -5,          /* Values would need 2^32 or more elements (TileOffset is 32-bit) */
-    SPDP_ERR_TIMEOUT = -6            /* a bounded device-side wait expired (device status word) */
+    SPDP_ERR_TIMEOUT = -6            /* reserved: a bounded device-side wait expired (no kernel waits today) */
 } spdp_status;
 
 /* Dynamic-pruning rule: which columns of W are fetched for this x (Sec. 2.2 "Dynamic Pruning",
@@ -117,8 +117,9 @@ SPDP_API spdp_status spdp_import_tiled_cbc(int64_t M, int64_t K, int pad_elems, 
  *             Every one of the M entries is written, also when no column is active (zeros).
  * Asynchronous on `stream`; allocates nothing and never synchronises.  Launches one kernel.
  * The summation order is fixed for a given handle, so repeated calls give identical bits.
- * Device-side problems (a bounded wait that expired) are recorded in the handle's device
- * status word, readable with spdp_last_device_status. */
+ * No CTA of the kernel ever waits for another one (the split-K combine is made of single atomic
+ * exchanges), so there is nothing on the device that can time out; the handle's device status word,
+ * readable with spdp_last_device_status, is reserved for device-side checks and stays 0. */
 SPDP_API spdp_status spdp_spmspv(spdp_handle h, const void* x_dev, spdp_dp_rule rule, float thr,
                         const void* mask_dev, void* y_dev, spdp_ydtype ydt, void* stream);
 

@@ -35,7 +35,7 @@ NOMINAL_HBM_GBS = 8000.0          # the "roughly 8 TB/s" the 70 % target is quot
 FALLBACK_HBM_GBS = 6650.0         # used only if MEASURED_PEAKS.json is absent
 # dram__bytes_read.sum + dram__bytes_write.sum of one spmspv launch on the default workload,
 # from the ncu capture summarised under profiles/.
-NCU_TRAFFIC_BYTES = {"c4": 183657216 + 4031232}      # profiles/spmspv_kernel_c4_ncu_full.md
+NCU_TRAFFIC_BYTES = {"c4": 183657728 + 4013568}      # profiles/spmspv_kernel_c4_ncu_full.md
 
 
 def make_workload(name: str):

@@ -164,3 +164,38 @@ def test_batch_active_sets_on_threshold_edges(S, thr):
             assert np.array_equal(Y[b], want), (thr, b)
     finally:
         S.spdp_free(h)
+
+
+def test_batch_in_a_cuda_graph_next_to_single_calls(S):
+    """The batch call only launches: captured with a single-vector call on the same handle and replayed."""
+    rng = np.random.Generator(np.random.PCG64(41))
+    M, K, B = 1500, 3000, 6
+    W = (rng.standard_normal((M, K)) * (rng.random((M, K)) < 0.45) * 0.05).astype(np.float16)
+    X = rng.standard_normal((B, K)).astype(np.float16)
+    rule, thr = O.DP_ABS_GT, 0.5
+    acts = np.stack([O.active_ref(X[b], rule, thr) for b in range(B)])
+    Y_ref, S_ref = O.spmspv_batch_ref(W, X, acts)
+    h = S.spdp_pack_tiled_cbc(dev(W))
+    try:
+        Xd = dev(X)
+        Y = torch.zeros((B, M), dtype=torch.float32, device="cuda")
+        y0 = torch.zeros(M, dtype=torch.float32, device="cuda")
+        S.spdp_spmspv_batch(h, Xd, rule, thr, Y)                       # warm-up outside the capture
+        S.spdp_spmspv(h, Xd[0], rule, thr, y0)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        side = torch.cuda.Stream()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(g, stream=side):
+                S.spdp_spmspv_batch(h, Xd, rule, thr, Y, stream=side.cuda_stream)
+                S.spdp_spmspv(h, Xd[0], rule, thr, y0, stream=side.cuda_stream)
+                S.spdp_spmspv_batch(h, Xd, rule, thr, Y, stream=side.cuda_stream)
+        for _ in range(3):
+            Y.fill_(float("nan"))
+            y0.fill_(float("nan"))
+            g.replay()
+            torch.cuda.synchronize()
+            check(Y.cpu().numpy(), Y_ref, S_ref)
+            check(y0.cpu().numpy()[None, :], Y_ref[:1], S_ref[:1])
+    finally:
+        S.spdp_free(h)

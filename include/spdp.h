@@ -15,6 +15,8 @@
  *  - A handle owns its packed arrays, its split-K workspace and a few staging buffers.  The
  *    workspace is per handle, so at most ONE spdp_spmspv per handle may be in flight; calls on
  *    one handle must be ordered (same stream, or events).  Different handles are independent.
+ *    A call that was aborted, or that overlapped another call on the same handle, can leave a partial
+ *    sum in the workspace; spdp_set_num_ctas (any value, also the current one) empties it again.
  *  - Format constants: column tile 256 x 1, GTile 256 x 16, four 64-bit bitmap words per column
  *    tile (Sec. 4.1); 16-byte padding of every column's values (Sec. 4.2.3).
  */
@@ -201,6 +203,17 @@ SPDP_API spdp_status spdp_unpack(spdp_handle h, void* W_dev_out, int64_t ldw, vo
 SPDP_API spdp_status spdp_active_columns(spdp_handle h, const void* x_dev, spdp_dp_rule rule, float thr,
                                 const void* mask_dev, void* bitmask_dev_out, void* count_dev_out,
                                 void* stream);
+
+/* Context measurements for the benchmark (the paper has no counterpart; they compute nothing).
+ * spdp_probe_stream_read reads the handle's Values array front to back with plain 16-byte loads;
+ * spdp_probe_gather reads exactly what one spdp_spmspv call with these arguments must fetch -- the
+ * ColInfo / TileOffset words of the active columns, their bitmaps and their padded values -- with
+ * plain loads and no decoding.  Both are asynchronous on `stream`, allocate nothing and write
+ * nothing the caller can see; the caller times them.  They give the speed of a contiguous read and
+ * the ceiling of the method's access pattern on this GPU, next to which the kernel is reported. */
+SPDP_API spdp_status spdp_probe_stream_read(spdp_handle h, void* stream);
+SPDP_API spdp_status spdp_probe_gather(spdp_handle h, const void* x_dev, spdp_dp_rule rule, float thr,
+                              const void* mask_dev, void* stream);
 
 /* Read (and clear) the handle's device status word: 0, or an spdp_status recorded by a kernel.
  * Synchronises the device. */

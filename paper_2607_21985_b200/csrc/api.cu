@@ -81,6 +81,9 @@ spdp_status build_partition(spdp_matrix* h, int num_ctas) {
     SPDP_CUDA_TRY(cudaMalloc(&h->workspace_batch, batch_workspace_bytes(P)));
     SPDP_CUDA_TRY(cudaMemset(h->workspace_batch, 0, batch_workspace_bytes(P)));
     h->workspace_bytes += batch_workspace_bytes(P);
+    // The memsets run on the legacy default stream, which a non-blocking stream does not wait for:
+    // the first spdp_spmspv on such a stream must find every tree node empty.
+    SPDP_CUDA_TRY(cudaDeviceSynchronize());
     return SPDP_OK;
 }
 
@@ -91,11 +94,12 @@ spdp_status finish_handle(spdp_matrix* h) {
     if (st != SPDP_OK) return st;
     st = configure_spmspv_batch_kernel();
     if (st != SPDP_OK) return st;
-    SPDP_CUDA_TRY(cudaMalloc(&h->status_word, sizeof(int)));
-    SPDP_CUDA_TRY(cudaMemset(h->status_word, 0, sizeof(int)));
+    SPDP_CUDA_TRY(cudaMalloc(&h->status_word, 2 * sizeof(int)));
+    SPDP_CUDA_TRY(cudaMemset(h->status_word, 0, 2 * sizeof(int)));
     SPDP_CUDA_TRY(cudaMalloc(&h->x_stage, h->K * sizeof(__half)));
     SPDP_CUDA_TRY(cudaMalloc(&h->mask_stage, ((h->K + 31) / 32) * sizeof(uint32_t)));
     SPDP_CUDA_TRY(cudaMalloc(&h->y_stage, h->M * sizeof(float)));
+    SPDP_CUDA_TRY(cudaDeviceSynchronize());     // the status word's memset, for callers on non-blocking streams
     return SPDP_OK;
 }
 
@@ -412,6 +416,20 @@ spdp_status spdp_active_columns(spdp_handle h, const void* x_dev, spdp_dp_rule r
     return launch_active_columns(h, static_cast<const __half*>(x_dev), rule, thr,
                                  static_cast<const uint32_t*>(mask_dev), static_cast<uint32_t*>(bitmask_dev_out),
                                  static_cast<int*>(count_dev_out), static_cast<cudaStream_t>(stream));
+}
+
+spdp_status spdp_probe_stream_read(spdp_handle h, void* stream) {
+    if (!valid(h)) return SPDP_ERR_INVALID_ARG;
+    return launch_probe_stream_read(h, static_cast<cudaStream_t>(stream));
+}
+
+spdp_status spdp_probe_gather(spdp_handle h, const void* x_dev, spdp_dp_rule rule, float thr, const void* mask_dev,
+                              void* stream) {
+    if (!valid(h) || x_dev == nullptr) return SPDP_ERR_INVALID_ARG;
+    if (!rule_ok(rule) || (rule == SPDP_DP_MASK && mask_dev == nullptr)) return SPDP_ERR_INVALID_ARG;
+    if (h->pad_elems != 8) return SPDP_ERR_UNSUPPORTED_SHAPE;
+    return launch_probe_gather(h, static_cast<const __half*>(x_dev), rule, thr, static_cast<const uint32_t*>(mask_dev),
+                               static_cast<cudaStream_t>(stream));
 }
 
 spdp_status spdp_last_device_status(spdp_handle h, int* out) {

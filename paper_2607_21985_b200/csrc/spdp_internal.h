@@ -37,7 +37,7 @@ struct spdp_matrix {
     int num_ctas;           // P
     float* workspace;       // device [P*256] split-K tree nodes, one row per CTA (all zero between calls)
     float* workspace_batch; // device [P*8*256] tree nodes of the small-batch call (all zero between calls)
-    int* status_word;       // device [1]
+    int* status_word;       // device [2]: the status word, and a sink word the benchmark probes may write
     int64_t workspace_bytes;
 
     // Staging for the host-vector entry point
@@ -94,6 +94,11 @@ int64_t batch_workspace_bytes(int num_ctas);
 spdp_status configure_spmspv_batch_kernel();   // per-device kernel attributes; idempotent
 spdp_status launch_spmspv_batch(const spdp_matrix* h, const __half* x, int64_t ldx, int batch, int rule, float thr,
                                 const uint32_t* mask, int64_t mask_stride, void* y, int64_t ldy, int ydt,
+                                cudaStream_t s);
+
+// probes.cu (context measurements for the benchmark)
+spdp_status launch_probe_stream_read(const spdp_matrix* h, cudaStream_t s);
+spdp_status launch_probe_gather(const spdp_matrix* h, const __half* x, int rule, float thr, const uint32_t* mask,
                                 cudaStream_t s);
 
 spdp_status launch_active_columns(const spdp_matrix* h, const __half* x, int rule, float thr,

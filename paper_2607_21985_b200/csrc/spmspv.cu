@@ -317,8 +317,12 @@ spmspv_kernel(const Params p) {
                         m |= (!(fabsf(hi) <= p.thr) ? 1u : 0u) << (2 * i + 1);
                     }
                 } else if (p.rule == SPDP_DP_MASK) {
-                    const int j0 = (v0 < vB0) ? jA0 + v0 : v0 - vB0;     // a multiple of 8
-                    m = (__ldg(p.mask + (j0 >> 5)) >> (j0 & 31)) & 0xFFu;
+                    // units of the padding between the two pieces hold no column: they must not touch
+                    // the mask (their word can lie one past its end)
+                    if (lim > 0) {
+                        const int j0 = (v0 < vB0) ? jA0 + v0 : v0 - vB0; // a multiple of 8
+                        m = (__ldg(p.mask + (j0 >> 5)) >> (j0 & 31)) & 0xFFu;
+                    }
                 } else {
                     m = 0xFFu;
                 }
@@ -547,9 +551,9 @@ __global__ void active_columns_kernel(const __half* __restrict__ x, int K, int r
 
 
 // ---- allocation-free variant: scratch in a file-scope device array --------------------------
-// Everything spdp_spmspv keeps in handle-owned allocations (the CTA ranges, the per-row-tile
-// tables, the arrival counters, the split-K partial sums) lives here instead, so the entry point
-// below never allocates.  One copy per device that loads the library, held until exit.
+// What spdp_spmspv keeps in handle-owned allocations (the device status word and the workspace of
+// split-K tree nodes, one row of 256 per CTA) lives here instead, so the entry point below never
+// allocates.  One copy per device that loads the library, held until exit.
 constexpr int kNoAllocMaxCtas = 512;
 
 struct NoAllocScratch {

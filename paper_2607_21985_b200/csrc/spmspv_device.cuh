@@ -2,6 +2,7 @@
 // shared-memory accesses with explicit state space, the work split and the split-K combine.
 #pragma once
 
+#include "spdp_hostdev.h"
 #include "spdp_internal.h"
 
 namespace spdp {
@@ -80,15 +81,8 @@ __device__ __forceinline__ const unsigned char* offset_wide(const unsigned char*
     return r;
 }
 
-// The work split: CTA c of num_ctas owns GTiles [range_begin(c), range_begin(c + 1)) of the row-major
-// GTile order.  NGT < 2^22 and num_ctas <= 1024 keep every product below 2^32.
-__device__ __forceinline__ unsigned range_begin(unsigned ngt, unsigned num_ctas, unsigned c) {
-    return (ngt * c) / num_ctas;
-}
-// The CTA whose range holds GTile g: ceil((g + 1) * num_ctas / NGT) - 1.
-__device__ __forceinline__ int range_owner(unsigned ngt, unsigned num_ctas, unsigned g) {
-    return static_cast<int>(((g + 1u) * num_ctas + ngt - 1u) / ngt) - 1;
-}
+using hostdev::range_begin;     // the work split lives in spdp_hostdev.h (shared with the host)
+using hostdev::range_owner;
 
 // A partial sum is kept in the workspace XOR this key, so that the all-zero word means "empty".
 // NaN sums are made canonical first, which keeps a stored word from ever being zero.

@@ -29,7 +29,7 @@ EXPORTS = (
     "spdp_pack_tiled_cbc", "spdp_pack_tiled_cbc_ex", "spdp_import_tiled_cbc", "spdp_spmspv",
     "spdp_spmspv_host", "spdp_spmspv_noalloc", "spdp_spmspv_batch", "spdp_free", "spdp_get_info", "spdp_export", "spdp_unpack",
     "spdp_active_columns", "spdp_last_device_status", "spdp_set_num_ctas", "spdp_last_cuda_error",
-    "spdp_status_string",
+    "spdp_status_string", "spdp_probe_stream_read", "spdp_probe_gather",
 )
 
 
@@ -74,6 +74,8 @@ def lib():
         L.spdp_active_columns.argtypes = [vp, vp, ci, cf, vp, vp, vp, vp]
         L.spdp_last_device_status.argtypes = [vp, ctypes.POINTER(ci)]
         L.spdp_set_num_ctas.argtypes = [vp, ci]
+        L.spdp_probe_stream_read.argtypes = [vp, vp]
+        L.spdp_probe_gather.argtypes = [vp, vp, ci, cf, vp, vp]
         for name in EXPORTS:
             getattr(L, name).restype = ci
         L.spdp_last_cuda_error.restype = ctypes.c_char_p
@@ -258,6 +260,17 @@ def spdp_last_device_status(h: int) -> int:
 
 def spdp_set_num_ctas(h: int, num_ctas: int) -> None:
     _check(lib().spdp_set_num_ctas(h, num_ctas), "spdp_set_num_ctas")
+
+
+def spdp_probe_stream_read(h: int, stream=None) -> None:
+    """Benchmark context: one contiguous read of the handle's Values array."""
+    _check(lib().spdp_probe_stream_read(h, _stream(stream)), "spdp_probe_stream_read")
+
+
+def spdp_probe_gather(h: int, x, rule: int, thr: float, mask=None, stream=None) -> None:
+    """Benchmark context: fetch what spdp_spmspv would fetch for this x, with plain loads and no decode."""
+    _check(lib().spdp_probe_gather(h, _dev_ptr(x, "x"), rule, float(thr), _dev_ptr(mask, "mask", True), _stream(stream)),
+           "spdp_probe_gather")
 
 
 def spdp_status_string(status: int) -> str:

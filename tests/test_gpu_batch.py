@@ -199,3 +199,36 @@ def test_batch_in_a_cuda_graph_next_to_single_calls(S):
             check(y0.cpu().numpy()[None, :], Y_ref[:1], S_ref[:1])
     finally:
         S.spdp_free(h)
+
+
+def test_batch_non_finite_values_follow_the_documented_reading(S):
+    """Where the batch call departs from the token-by-token definition, pinned so that it cannot drift:
+    a token that skips a column enters it with x = 0, so (a) an Inf weight in a column tile that is fetched
+    for ANOTHER token gives NaN (0 * Inf) in that row for the token that skips the column -- and only
+    there; (b) a NaN activation of a kept column reaches every row of that token (0 * NaN through the
+    zeros of the fetched tiles).  Tokens without such values, and all other rows, follow the definition."""
+    rng = np.random.Generator(np.random.PCG64(55))
+    M, K, B = 300, 64, 4
+    W = (rng.standard_normal((M, K)) * (rng.random((M, K)) < 0.5) * 0.05).astype(np.float16)
+    W[5, 50] = np.inf
+    X = rng.standard_normal((B, K)).astype(np.float16)
+    X[0, 50] = 1.0            # token 0 keeps column 50
+    X[1, 50] = 0.0            # token 1 skips it (thr = 0 skips exact zeros), token 0 makes it fetched
+    X[2, 50] = 0.0
+    X[2, 60] = np.nan         # token 2 keeps a NaN activation
+    X[3, 50] = 2.0
+    rule, thr = O.DP_ABS_GT, 0.0
+    acts = np.stack([O.active_ref(X[b], rule, thr) for b in range(B)])
+    Y_ref, S_ref = O.spmspv_batch_ref(W, X, acts)
+    h = S.spdp_pack_tiled_cbc(dev(W))
+    try:
+        Y = run_batch(S, h, X, rule, thr, M)
+    finally:
+        S.spdp_free(h)
+    rows = np.arange(M) != 5
+    assert Y[0, 5] == np.inf and Y[3, 5] == np.inf                    # kept: Inf * x, as the definition
+    check(Y[[0, 3]][:, rows], Y_ref[[0, 3]][:, rows], S_ref[[0, 3]][:, rows])
+    assert np.isnan(Y[1, 5]) and np.isfinite(Y_ref[1, 5])             # (a): 0 * Inf where the definition omits
+    check(Y[1:2, rows], Y_ref[1:2, rows], S_ref[1:2, rows])           # ... and nowhere else
+    assert np.isnan(Y[2]).all()                                       # (b): every row of the token
+    assert np.isnan(Y_ref[2][O.is_nonzero(W[:, 60])]).all() and not np.isnan(Y_ref[2][~O.is_nonzero(W[:, 60]) & rows]).any()

@@ -370,3 +370,81 @@ def test_scaled_down_benchmark_layers(S, make):
         check_y(gpu_spmspv(S, h, w.x, w.rule, w.thr, w.M, torch.float32), y_ref, S_ref)
     finally:
         S.spdp_free(h)
+
+
+# ------------------------------------------------------------------------------------------
+# the single-vector kernel's own DP test (it lists the active columns itself, 8 per thread)
+# ------------------------------------------------------------------------------------------
+def _striped_identity(M, K):
+    """One stored 1.0 per column, at row j % M: y then shows every column's decision by itself."""
+    W = torch.zeros((M, K), dtype=torch.float16, device="cuda")
+    j = torch.arange(K, device="cuda")
+    W[j % M, j] = 1.0
+    return W
+
+
+@pytest.mark.parametrize("thr", [0.5, 0.50006103515625, 0.3, 0.0, -0.0, -1.0, 1e-10, 70000.0, float("inf"),
+                                 float("-inf"), float("nan"), 6.1e-5, 5.96e-8])
+def test_spmspv_active_set_on_threshold_edges(S, thr):
+    """Values at, just below and just above the threshold (in fp16 steps), zeros of both signs, subnormals,
+    the largest finite values, NaN and both infinities, under finite, infinite and NaN thresholds: the
+    kernel's in-line DP test must take the oracle's decision for every one.  Also with x only 2-byte
+    aligned (the plain-load path) and with the probes astride column 8192, where a CTA that owns a long
+    stretch of one row tile ends one list of columns and begins the next."""
+    base = np.float16(thr) if np.isfinite(thr) and abs(thr) < 65504 else np.float16(1.0)
+    around = np.array([base, np.nextafter(base, np.float16(np.inf)), np.nextafter(base, np.float16(-np.inf)),
+                       -base, 0.0, -0.0, 6e-8, -6e-8, 6.1e-5, 65504, -65504, 0.25, 0.5, 0.75,
+                       np.nan, np.inf, -np.inf], dtype=np.float16)
+    rng = np.random.Generator(np.random.PCG64(78))
+    for K, ctas, shift in ((64, 0, 0), (16400, 1, 0), (16400, 3, 1), (16400, 0, 3)):
+        M = min(K, 256)
+        first = 0 if K == 64 else 8192 - 7                     # probes astride the end of the first list
+        x = np.zeros(K, dtype=np.float16)
+        x[first:first + len(around)] = rng.permutation(around)
+        a = O.active_ref(x, O.DP_ABS_GT, thr)
+        want = np.zeros(M, dtype=np.float32)
+        for p in range(first, first + len(around)):
+            if a[p]:
+                want[p % M] = np.float32(x[p])
+        h = S.spdp_pack_tiled_cbc(_striped_identity(M, K))
+        try:
+            if ctas:
+                S.spdp_set_num_ctas(h, ctas)
+            buf = torch.zeros(K + 8, dtype=torch.float16, device="cuda")
+            xs = buf[shift:shift + K]
+            xs.copy_(dev(x))
+            y = torch.full((M,), float("nan"), dtype=torch.float32, device="cuda")
+            S.spdp_spmspv(h, xs, O.DP_ABS_GT, thr, y)
+            torch.cuda.synchronize()
+            assert np.array_equal(y.cpu().numpy(), want, equal_nan=True), (thr, K, ctas, shift)
+            bits, cnt = gpu_active(S, h, x, O.DP_ABS_GT, thr, K)
+            assert np.array_equal(bits, O.active_to_words(a)) and cnt == int(a.sum())
+        finally:
+            S.spdp_free(h)
+
+
+def test_mask_rule_with_the_mask_at_the_end_of_its_allocation(S):
+    """Explicit mask whose last word is the last word of its buffer, on shapes where a CTA's range starts at
+    an odd GTile column (the list then has padding units between its two pieces, which must not read the
+    mask), and a first call issued on a side stream right after packing."""
+    for M, K, ctas in ((512, 4096, 3), (768, 4128, 7), (1024, 2080, 5)):
+        rw, rx = WL._rngs(40 + ctas)
+        W = WL.prune_global_magnitude(WL.normal_weights(rw, M, K), 0.5).astype(np.float16)
+        x = rx.standard_normal(K, dtype=np.float32).astype(np.float16)
+        m = rx.random(K) < 0.5
+        y_ref, S_ref = O.spmspv_ref(W, x, m)
+        words = O.active_to_words(m)
+        arena = torch.zeros(4096 + len(words), dtype=torch.int32, device="cuda")
+        md = arena[4096:]
+        md.copy_(dev(words))
+        side = torch.cuda.Stream()
+        with torch.cuda.stream(side):
+            h = S.spdp_pack_tiled_cbc(dev(W), stream=side)
+            try:
+                S.spdp_set_num_ctas(h, ctas)
+                y = torch.full((M,), float("nan"), dtype=torch.float32, device="cuda")
+                S.spdp_spmspv(h, dev(x), O.DP_MASK, 0.0, y, mask=md, stream=side)
+                side.synchronize()
+                check_y(y.cpu().numpy().astype(np.float64), y_ref, S_ref)
+            finally:
+                S.spdp_free(h)

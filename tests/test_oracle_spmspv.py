@@ -190,3 +190,16 @@ def test_batch_union_and_bytes():
     assert O.active_bytes_batch(p, same) == O.active_bytes(p, acts[0]) + (B - 1) * (2 * K + 2 * M)
     assert O.active_bytes_batch(p, acts) >= max(O.active_bytes(p, a) for a in acts)
     assert O.active_bytes_batch(p, acts[:1]) == O.active_bytes(p, acts[0])
+
+
+def test_tolerance_is_the_stated_bound_on_literal_numbers():
+    """The parity gate of every y comparison is |y - y_ref| <= 1e-3 * S + 1e-5 (the bound the task states):
+    literal values, so that a looser constant (1e-2, 1e-4 absolute) fails here."""
+    got = O.tolerance(np.array([0.0, 1.0, 250.0, 1e-2, 4.0e3]))
+    want = [1e-5, 1.01e-3, 0.25001, 2e-5, 4.00001]
+    assert got.dtype == np.float64 and got.shape == (5,)
+    assert np.allclose(got, want, rtol=1e-14, atol=0.0)
+    assert O.tolerance(2.0) == pytest.approx(2.01e-3, rel=1e-14)
+    # an error of twice the bound is refused, one of half the bound passes (how the tests use it)
+    S = np.array([3.0])
+    assert not (np.array([2 * 3.01e-3]) <= O.tolerance(S)).any() and (np.array([0.5 * 3.01e-3]) <= O.tolerance(S)).all()

@@ -208,8 +208,10 @@ SPDP_API spdp_status spdp_active_columns(spdp_handle h, const void* x_dev, spdp_
  * spdp_probe_stream_read reads the handle's Values array front to back with plain 16-byte loads;
  * spdp_probe_gather reads exactly what one spdp_spmspv call with these arguments must fetch -- the
  * ColInfo / TileOffset words of the active columns, their bitmaps and their padded values -- with
- * plain loads and no decoding.  Both are asynchronous on `stream`, allocate nothing and write
- * nothing the caller can see; the caller times them.  They give the speed of a contiguous read and
+ * plain loads and no decoding (its first call, and any call with other arguments, first builds the
+ * list of those tiles in a scratch buffer it allocates; repeated calls with the same pointers reuse
+ * the list, so time the repeats).  Both are asynchronous on `stream` and write nothing the caller can
+ * see; the caller times them.  They give the speed of a contiguous read and
  * the ceiling of the method's access pattern on this GPU, next to which the kernel is reported. */
 SPDP_API spdp_status spdp_probe_stream_read(spdp_handle h, void* stream);
 SPDP_API spdp_status spdp_probe_gather(spdp_handle h, const void* x_dev, spdp_dp_rule rule, float thr,

@@ -31,6 +31,8 @@ void release(spdp_matrix* h) {
     cudaFree(h->x_stage);
     cudaFree(h->mask_stage);
     cudaFree(h->y_stage);
+    cudaFree(h->probe_items);
+    cudaFree(h->probe_count);
     if (h->host_graph != nullptr) cudaGraphExecDestroy(h->host_graph);
     if (h->capture_stream != nullptr) cudaStreamDestroy(h->capture_stream);
     h->magic = 0;

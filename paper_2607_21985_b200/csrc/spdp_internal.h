@@ -59,6 +59,17 @@ struct spdp_matrix {
     HostCallKey host_graph_key;     // arguments the graph below was recorded with
     cudaGraphExec_t host_graph;     // null: none
     cudaStream_t capture_stream;    // private stream used only to record that graph
+
+    // Benchmark probe (spdp_probe_gather): the list of active column tiles it reads, built on first use.
+    struct ProbeKey {
+        const void* x;
+        const void* mask;
+        int rule;
+        float thr;
+    };
+    void* probe_items;              // device uint2[R*K], null until the probe is first called
+    void* probe_count;              // device uint64[1]
+    ProbeKey probe_key;
 };
 
 namespace spdp {
@@ -98,7 +109,7 @@ spdp_status launch_spmspv_batch(const spdp_matrix* h, const __half* x, int64_t l
 
 // probes.cu (context measurements for the benchmark)
 spdp_status launch_probe_stream_read(const spdp_matrix* h, cudaStream_t s);
-spdp_status launch_probe_gather(const spdp_matrix* h, const __half* x, int rule, float thr, const uint32_t* mask,
+spdp_status launch_probe_gather(spdp_matrix* h, const __half* x, int rule, float thr, const uint32_t* mask,
                                 cudaStream_t s);
 
 spdp_status launch_active_columns(const spdp_matrix* h, const __half* x, int rule, float thr,

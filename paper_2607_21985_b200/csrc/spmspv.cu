@@ -66,6 +66,7 @@ struct Params {
     int num_ctas;
     float* workspace;       // [num_ctas][256] tree nodes of the split-K combine, all zero between calls
     int* status;
+    int64_t values_len;     // elements of Values (the checked build holds every fetch against it)
 };
 
 struct __align__(128) Smem {
@@ -173,6 +174,10 @@ __device__ __forceinline__ void finish_row_tile(const Params& p, int r, const fl
     if (row >= p.M) return;
     const int q0 = range_owner(p, static_cast<unsigned>(r) * p.C);                 // first and last CTA feeding row tile r
     const int nseg = range_owner(p, static_cast<unsigned>(r + 1) * p.C - 1u) - q0 + 1;
+    if (!SPDP_CHECK(p.status, q0, nseg, p.num_ctas, kSiteTreeNodes) ||
+        !SPDP_CHECK(p.status, static_cast<int>(blockIdx.x) - q0, 1, nseg, kSiteTreeNodes) ||
+        !SPDP_CHECK(p.status, row, 1, p.M, kSiteOutputRow))
+        return;
     if (tree_combine(part, reinterpret_cast<unsigned*>(p.workspace) + tt, kTileM, q0, nseg,
                      static_cast<int>(blockIdx.x) - q0))
         store_y(p.y, p.ydt, row, part);
@@ -377,8 +382,16 @@ spmspv_kernel(const Params p) {
 #pragma unroll
                     for (int b = 0; b < 8; ++b) {
                         if ((m >> b) & 1u) {
-                            sm.rec[item] = make_uint2(to + (ci[b] >> 16), ((slot0 + b) << 6) | (((ci[b] & 0xFFFFu) + 7u) >> 3));
-                            sm.xact[item] = static_cast<unsigned short>((b & 1) ? (xw[b >> 1] >> 16) : (xw[b >> 1] & 0xFFFFu));
+                            const unsigned start = to + (ci[b] >> 16), pieces = ((ci[b] & 0xFFFFu) + 7u) >> 3;
+                            const bool ok = SPDP_CHECK(p.status, item, 1, kChunkCols, kSiteRecordIndex);
+                            if (ok && SPDP_CHECK(p.status, start, 8u * pieces, p.values_len, kSiteValuesSpan) &&
+                                SPDP_CHECK(p.status, 0, pieces, 32, kSitePieces) &&
+                                SPDP_CHECK(p.status, slot0 + b, 1, p.NGT * kTileK, kSiteBitmapSlot)) {
+                                sm.rec[item] = make_uint2(start, ((slot0 + b) << 6) | pieces);
+                                sm.xact[item] = static_cast<unsigned short>((b & 1) ? (xw[b >> 1] >> 16) : (xw[b >> 1] & 0xFFFFu));
+                            } else if (ok) {
+                                sm.rec[item] = make_uint2(0u, kNullRec);       // checked build only: the tile is left out
+                            }
                             ++item;
                         }
                     }
@@ -611,6 +624,7 @@ spdp_status launch_spmspv(const spdp_matrix* h, const __half* x, int rule, float
     p.num_ctas = h->num_ctas;
     p.workspace = h->workspace;
     p.status = h->status_word;
+    p.values_len = h->values_len;
     return launch_kernel(p, h->num_ctas, s);
 }
 
@@ -664,6 +678,7 @@ spdp_status launch_spmspv_noalloc(const uint32_t* tileoffset, const uint32_t* co
     p.num_ctas = P;
     p.workspace = sc->workspace;            // addresses inside the device array (no host dereference)
     p.status = &sc->status;
+    p.values_len = int64_t(1) << 40;        // the caller owns Values; its length is not known here
     return launch_kernel(p, P, s);
 }
 

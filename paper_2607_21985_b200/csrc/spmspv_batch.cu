@@ -59,6 +59,8 @@ struct Params {
     int64_t NGT;
     int num_ctas;
     float* workspace;           // [num_ctas][kBT][256] tree nodes, all zero between calls
+    int* status;
+    int64_t values_len;         // elements of Values (the checked build holds every fetch against it)
 };
 
 struct __align__(128) Smem {
@@ -289,7 +291,16 @@ spmspv_batch_kernel(const Params p) {
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
                     if ((m >> k) & 1u) {
-                        sm.rec[item] = make_uint2(to + (ci[k] >> 16), ((slot0 + k) << 6) | (((ci[k] & 0xFFFFu) + 7u) >> 3));
+                        const unsigned start = to + (ci[k] >> 16), pieces = ((ci[k] & 0xFFFFu) + 7u) >> 3;
+                        const bool rec_ok = SPDP_CHECK(p.status, item, 1, kChunkCols, kSiteRecordIndex) &&
+                                            SPDP_CHECK(p.status, start, 8u * pieces, p.values_len, kSiteValuesSpan) &&
+                                            SPDP_CHECK(p.status, 0, pieces, 32, kSitePieces) &&
+                                            SPDP_CHECK(p.status, slot0 + k, 1, p.NGT * kTileK, kSiteBitmapSlot);
+                        if (!SPDP_CHECK(p.status, item, 1, kChunkCols, kSiteRecordIndex)) {
+                            ++item;
+                            continue;
+                        }
+                        sm.rec[item] = rec_ok ? make_uint2(start, ((slot0 + k) << 6) | pieces) : make_uint2(0u, kNullRec);
                         uint4 xr;
                         unsigned* xo = reinterpret_cast<unsigned*>(&xr);
 #pragma unroll
@@ -405,7 +416,8 @@ spmspv_batch_kernel(const Params p) {
             }
             // The four outputs walk the same tree (same segments); their exchanges at a level are
             // issued together, so the walk costs one round trip per level, not four.
-            if (tok < p.batch) {
+            if (tok < p.batch && SPDP_CHECK(p.status, q0, nseg, p.num_ctas, kSiteTreeNodes) &&
+                SPDP_CHECK(p.status, static_cast<int>(blockIdx.x) - q0, 1, nseg, kSiteTreeNodes)) {
                 unsigned* nodes = reinterpret_cast<unsigned*>(p.workspace) + tok * kTileM + rr;
                 const int64_t row0 = static_cast<int64_t>(r) * kTileM + rr;
                 bool alive[4];
@@ -485,6 +497,8 @@ spdp_status launch_spmspv_batch(const spdp_matrix* h, const __half* x, int64_t l
     p.NGT = h->NGT;
     p.num_ctas = h->num_ctas;
     p.workspace = h->workspace_batch;
+    p.status = h->status_word;
+    p.values_len = h->values_len;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(h->num_ctas));
     cfg.blockDim = dim3(kThreads);

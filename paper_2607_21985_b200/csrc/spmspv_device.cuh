@@ -84,6 +84,31 @@ __device__ __forceinline__ const unsigned char* offset_wide(const unsigned char*
 using hostdev::range_begin;     // the work split lives in spdp_hostdev.h (shared with the host)
 using hostdev::range_owner;
 
+// Checked build (-DSPDP_CHECKED): every record the kernels derive from the packed arrays (where a
+// column tile's values start, how many 16-byte pieces they are, which bitmap slot they belong to,
+// where the record goes) and every split-K node they are about to touch is held against its
+// array's size first.  A violation stores check_code(site) in the status word (the first one
+// wins) and the access is skipped: the tile is left out, the row is not stored.  Nothing traps and
+// nothing asserts; it is the stand-in for a memory checker on hosts that have none.
+#ifdef SPDP_CHECKED
+__device__ __forceinline__ bool checked_span(int* status, uint64_t first, uint64_t count, uint64_t limit, int site) {
+    if (hostdev::span_ok(first, count, limit)) return true;
+    atomicCAS(status, 0, hostdev::check_code(site));
+    return false;
+}
+#define SPDP_CHECK(status, first, count, limit, site) \
+    ::spdp::dev::checked_span((status), static_cast<uint64_t>(first), static_cast<uint64_t>(count), static_cast<uint64_t>(limit), (site))
+#else
+#define SPDP_CHECK(status, first, count, limit, site) true
+#endif
+// Sites of the checks (the number a violation reports, as check_code(site)).
+constexpr int kSiteRecordIndex = 1;     // record index inside the shared-memory list
+constexpr int kSiteValuesSpan = 2;      // a column tile's padded values inside Values
+constexpr int kSitePieces = 3;          // at most 32 16-byte pieces per column tile
+constexpr int kSiteBitmapSlot = 4;      // column slot inside Bitmap / ColInfo
+constexpr int kSiteTreeNodes = 5;       // split-K segments of a row tile inside the workspace
+constexpr int kSiteOutputRow = 6;       // output row inside y
+
 // A partial sum is kept in the workspace XOR this key, so that the all-zero word means "empty".
 // NaN sums are made canonical first, which keeps a stored word from ever being zero.
 constexpr unsigned kNodeKey = 0xFFC0DEADu;

@@ -319,6 +319,16 @@ def active_bytes_batch(p: dict, actives, y_bytes_per_elem: int = 2) -> int:
     return one + (B - 1) * (2 * p["K"] + y_bytes_per_elem * p["M"])
 
 
+def spmm_ref(W, X):
+    """Prefill product on the statically pruned matrix alone (Sec. 4.3, SPDP-SpMM: N tokens, static
+    pruning only, no dynamic pruning): Y[n][i] = sum_j W[i][j] * X[n][j] in fp64 over the dense masked
+    matrix, and the error scale S[n][i] = sum_j |W[i][j] * X[n][j]|.  X is [N][K] (one token per row),
+    Y and S are float64 [N][M]."""
+    Wd = as_f64(W)
+    Xd = as_f64(X)
+    return Xd @ Wd.T, np.abs(Xd) @ np.abs(Wd).T
+
+
 def tolerance(S) -> np.ndarray:
     """Per-output bound of the parity gate: 1e-3 * S[i] + 1e-5."""
     return 1e-3 * np.asarray(S, dtype=np.float64) + 1e-5

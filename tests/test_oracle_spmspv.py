@@ -203,3 +203,45 @@ def test_tolerance_is_the_stated_bound_on_literal_numbers():
     # an error of twice the bound is refused, one of half the bound passes (how the tests use it)
     S = np.array([3.0])
     assert not (np.array([2 * 3.01e-3]) <= O.tolerance(S)).any() and (np.array([0.5 * 3.01e-3]) <= O.tolerance(S)).all()
+
+
+# ---- prefill product (Sec. 4.3): static pruning only, N tokens ----
+def test_spmm_ref_one_token_is_the_decode_definition_without_dp():
+    w = WL.config2(300, 200, seed=3)
+    rng = np.random.Generator(np.random.PCG64(8))
+    X = rng.standard_normal((3, w.K)).astype(np.float16)
+    Y, S = O.spmm_ref(w.W, X)
+    for n in range(3):
+        y1, s1 = O.spmspv_ref(w.W, X[n], np.ones(w.K, bool))       # DP_NONE: every column active
+        assert np.array_equal(Y[n], y1) and np.array_equal(S[n], s1)
+
+
+def test_spmm_ref_against_explicit_loops_on_integers():
+    rng = np.random.Generator(np.random.PCG64(9))
+    M, K, N = 37, 29, 5
+    W = rng.integers(-6, 7, (M, K)).astype(np.float16)
+    W[rng.random((M, K)) < 0.5] = 0
+    X = rng.integers(-5, 6, (N, K)).astype(np.float16)
+    Y, S = O.spmm_ref(W, X)
+    for n in range(N):
+        for i in range(M):
+            acc = 0
+            sc = 0
+            for j in range(K):
+                t = int(W[i, j]) * int(X[n, j])
+                acc += t
+                sc += abs(t)
+            assert Y[n, i] == acc and S[n, i] == sc                 # exact: small integers
+    # a transposed operand or a swapped index would not survive a non-square, non-symmetric case
+    assert Y.shape == (N, M)
+
+
+def test_spmm_ref_from_packed_arrays_equals_dense():
+    w = WL.config1(512, 96, seed=5)
+    rng = np.random.Generator(np.random.PCG64(10))
+    X = rng.standard_normal((7, w.K)).astype(np.float16)
+    back = O.unpack_ref(O.pack_fast(w.W))
+    Ya, _ = O.spmm_ref(w.W, X)
+    Yb, _ = O.spmm_ref(back, X)
+    assert np.array_equal(Ya, Yb)
+    assert np.allclose(Ya, X.astype(np.float64) @ w.W.astype(np.float64).T, rtol=0, atol=0)   # cross-check only

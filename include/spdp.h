@@ -145,6 +145,23 @@ SPDP_API spdp_status spdp_spmspv_batch(spdp_handle h, const void* x_dev, int64_t
                               float thr, const void* mask_dev, int64_t mask_stride, void* y_dev, int64_t ldy,
                               spdp_ydtype ydt, void* stream);
 
+/* Prefill product on the same packed handle (Sec. 4.3, SPDP-SpMM): Y[n] = W_sp * X[n] for N tokens,
+ * static pruning only (no dynamic pruning: every column is fetched once per block of tokens).
+ * The column tiles are decoded from Tiled-CBC into dense fp16 operand tiles in shared memory (what
+ * the paper's layout-alignment stage does for its tensor-core path), the contraction runs on the
+ * 5th-generation tensor cores (tcgen05.mma, fp16 inputs, fp32 accumulation in tensor memory).
+ *   X_dev   fp16 [N][ldx], device, one token per row, ldx >= K elements between tokens; X_dev must
+ *           be 16-byte aligned and ldx a multiple of 8 (the tiles are copied in 16-byte pieces),
+ *           else SPDP_ERR_INVALID_ARG.
+ *   N       >= 1 tokens.
+ *   Y_dev   [N][ldy] of ydt, device, ldy >= M elements between tokens; all N*M entries are written.
+ * Asynchronous on `stream`, allocates nothing, launches one kernel; no split along K, so no
+ * workspace is touched and calls on one handle may overlap.  The waits inside the kernel (on the
+ * tensor cores' completion barrier) are bounded; one that runs out records SPDP_ERR_TIMEOUT in the
+ * handle's status word and the CTA leaves its outputs unwritten. */
+SPDP_API spdp_status spdp_spmm(spdp_handle h, const void* X_dev, int64_t N, int64_t ldx, void* Y_dev, int64_t ldy,
+                      spdp_ydtype ydt, void* stream);
+
 /* Same product with HOST vectors (Sec. 4.2): copies x_host (fp16 [K], ideally pinned) to a
  * staging buffer of the handle, runs spdp_spmspv, copies y back into y_host ([M] of ydt) and
  * synchronises `stream`.  mask_host is uint32[ceil(K/32)] or NULL.  When the same pinned buffers and

@@ -96,6 +96,8 @@ spdp_status finish_handle(spdp_matrix* h) {
     if (st != SPDP_OK) return st;
     st = configure_spmspv_batch_kernel();
     if (st != SPDP_OK) return st;
+    st = configure_spmm_kernel();
+    if (st != SPDP_OK) return st;
     SPDP_CUDA_TRY(cudaMalloc(&h->status_word, 2 * sizeof(int)));
     SPDP_CUDA_TRY(cudaMemset(h->status_word, 0, 2 * sizeof(int)));
     SPDP_CUDA_TRY(cudaMalloc(&h->x_stage, h->K * sizeof(__half)));
@@ -300,6 +302,20 @@ spdp_status spdp_spmspv_batch(spdp_handle h, const void* x_dev, int64_t ldx, int
         return SPDP_OK;
     }
     return launch_spmspv_batch(h, x, ldx, batch, rule, thr, mask, mask_stride, y_dev, ldy, ydt, s);
+}
+
+spdp_status spdp_spmm(spdp_handle h, const void* X_dev, int64_t N, int64_t ldx, void* Y_dev, int64_t ldy,
+                      spdp_ydtype ydt, void* stream) {
+    if (!valid(h) || X_dev == nullptr || Y_dev == nullptr) return SPDP_ERR_INVALID_ARG;
+    if (N < 1 || N > (int64_t(1) << 24) || ldx < h->K || ldy < h->M) return SPDP_ERR_INVALID_ARG;
+    if (ydt != SPDP_Y_F16 && ydt != SPDP_Y_F32) return SPDP_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(X_dev) & 15u) || (ldx & 7) ||
+        (reinterpret_cast<uintptr_t>(Y_dev) & (ydt == SPDP_Y_F32 ? 3u : 1u)))
+        return SPDP_ERR_INVALID_ARG;
+    if (h->pad_elems != 8) return SPDP_ERR_UNSUPPORTED_SHAPE;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev != h->device) return SPDP_ERR_INVALID_ARG;   // wrong current device
+    return launch_spmm(h, static_cast<const __half*>(X_dev), N, ldx, Y_dev, ldy, ydt, static_cast<cudaStream_t>(stream));
 }
 
 spdp_status spdp_spmspv_noalloc(const void* tileoffset_dev, const void* colinfo_dev, const void* bitmap_dev,

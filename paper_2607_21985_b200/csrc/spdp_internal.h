@@ -107,6 +107,11 @@ spdp_status launch_spmspv_batch(const spdp_matrix* h, const __half* x, int64_t l
                                 const uint32_t* mask, int64_t mask_stride, void* y, int64_t ldy, int ydt,
                                 cudaStream_t s);
 
+// spmm.cu
+spdp_status configure_spmm_kernel();            // per-device kernel attributes; idempotent
+spdp_status launch_spmm(const spdp_matrix* h, const __half* X, int64_t N, int64_t ldx, void* Y, int64_t ldy, int ydt,
+                        cudaStream_t s);
+
 // probes.cu (context measurements for the benchmark)
 spdp_status launch_probe_stream_read(const spdp_matrix* h, cudaStream_t s);
 spdp_status launch_probe_gather(spdp_matrix* h, const __half* x, int rule, float thr, const uint32_t* mask,

@@ -29,7 +29,7 @@ EXPORTS = (
     "spdp_pack_tiled_cbc", "spdp_pack_tiled_cbc_ex", "spdp_import_tiled_cbc", "spdp_spmspv",
     "spdp_spmspv_host", "spdp_spmspv_noalloc", "spdp_spmspv_batch", "spdp_free", "spdp_get_info", "spdp_export", "spdp_unpack",
     "spdp_active_columns", "spdp_last_device_status", "spdp_set_num_ctas", "spdp_last_cuda_error",
-    "spdp_status_string", "spdp_probe_stream_read", "spdp_probe_gather",
+    "spdp_status_string", "spdp_probe_stream_read", "spdp_probe_gather", "spdp_spmm",
 )
 
 
@@ -74,6 +74,7 @@ def lib():
         L.spdp_active_columns.argtypes = [vp, vp, ci, cf, vp, vp, vp, vp]
         L.spdp_last_device_status.argtypes = [vp, ctypes.POINTER(ci)]
         L.spdp_set_num_ctas.argtypes = [vp, ci]
+        L.spdp_spmm.argtypes = [vp, vp, i64, i64, vp, i64, ci, vp]
         L.spdp_probe_stream_read.argtypes = [vp, vp]
         L.spdp_probe_gather.argtypes = [vp, vp, ci, cf, vp, vp]
         for name in EXPORTS:
@@ -213,6 +214,22 @@ def spdp_spmspv_batch(h: int, X, rule: int, thr: float, Y, mask=None, stream=Non
                                  None if mask is None else mask.data_ptr(), mstride, Y.data_ptr(), ldy, ydt,
                                  _stream(stream))
     _check(st, "spdp_spmspv_batch")
+
+
+def spdp_spmm(h: int, X, Y, stream=None) -> None:
+    """Prefill call: X fp16 CUDA [N][K] (rows may be strided), Y fp16 or fp32 CUDA [N][M]."""
+    import torch
+    if X.dim() != 2 or Y.dim() != 2 or X.shape[0] != Y.shape[0] or not X.is_cuda or not Y.is_cuda:
+        raise ValueError("X must be CUDA [N][K] and Y CUDA [N][M]")
+    if Y.dtype not in (torch.float16, torch.float32) or X.dtype != torch.float16:
+        raise ValueError("X must be fp16 and Y fp16 or fp32")
+    if X.stride(1) != 1 or Y.stride(1) != 1:
+        raise ValueError("the last dimension of X and Y must be contiguous")
+    N = int(X.shape[0])
+    ldx = int(X.stride(0)) if N > 1 else max(int(X.shape[1]), int(X.stride(0)))
+    ldy = int(Y.stride(0)) if N > 1 else max(int(Y.shape[1]), int(Y.stride(0)))
+    ydt = SPDP_Y_F32 if Y.dtype == torch.float32 else SPDP_Y_F16
+    _check(lib().spdp_spmm(h, X.data_ptr(), N, ldx, Y.data_ptr(), ldy, ydt, _stream(stream)), "spdp_spmm")
 
 
 def spdp_free(h) -> None:

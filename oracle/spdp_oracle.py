@@ -329,6 +329,133 @@ def spmm_ref(W, X):
     return Xd @ Wd.T, np.abs(Xd) @ np.abs(Wd).T
 
 
+# --------------------------------------------------------------------------------------
+# Low-bit Values payload (Sec. 5.1: 4-bit round-to-nearest weights, applied in the order static
+# pruning -> quantisation -> dynamic pruning; Sec. 6: Values are stored apart from the sparsity
+# metadata, so they can be low-bit).  The paper fixes no packed layout for it; this one keeps
+# TileOffset / ColInfo / Bitmap as they are and replaces Values by 4-bit codes plus one fp16 scale
+# per column tile:
+#   scale  = fp16( max|w| of the column tile's stored values / 7 )          (computed in fp32)
+#   q      = clamp( rint( w / scale ), -7, 7 )   in fp32, ties to even;  q = 0 where scale == 0
+#   code   = q + 8   (1..15; 0 never encodes a stored value)
+#   Codes  : per column tile its n codes in row order, two per byte (even rank = low nibble),
+#            zero-padded to 32 codes (16 bytes); TileOffset and ColInfo offsets count CODES
+#   weight = (code - 8) * scale
+# Non-finite weights are outside this variant (their codes are unspecified).
+# --------------------------------------------------------------------------------------
+Q4_PAD = 32
+
+
+def quantise_q4_ref(vals):
+    """One column tile's stored values (fp16) -> (scale as fp16 bits, codes uint8 in 1..15)."""
+    v32 = as_bits(np.asarray(vals)).view(np.float16).astype(np.float32)
+    if v32.size == 0:
+        return np.uint16(0), np.zeros(0, np.uint8)
+    s16 = (np.max(np.abs(v32)) / np.float32(7.0)).astype(np.float16)
+    s32 = np.float32(s16)
+    if s32 == 0:
+        q = np.zeros(v32.shape, np.int32)
+    else:
+        q = np.clip(np.rint(v32 / s32), -7, 7).astype(np.int32)
+    return s16.view(np.uint16), (q + 8).astype(np.uint8)
+
+
+def pack_q4_ref(W) -> dict:
+    """Dense pruned fp16 W -> the 4-bit variant of Tiled-CBC, written as the definition (loops over
+    GTiles and columns).  Returns dict(M, K, pad_elems=32, tileoffset u32[NGT+1] (in codes),
+    colinfo u32[NGT*16] (offset in codes << 16 | nnz), bitmap u64[NGT*64], codes u8[TileOffset[NGT]/2],
+    scales u16[NGT*16] (fp16 bits), nnz)."""
+    Wb = as_bits(W)
+    M, K = Wb.shape
+    R, C, NGT = grid(M, K)
+    base = pack_ref(Wb, pad_elems=Q4_PAD)                  # same bitmap; offsets with the 32-code padding
+    scales = np.zeros(NGT * TILE_K, dtype=np.uint16)
+    nibbles = np.zeros(int(base["tileoffset"][NGT]), dtype=np.uint8)
+    for g in range(NGT):
+        for cc in range(TILE_K):
+            slot = g * TILE_K + cc
+            ci = int(base["colinfo"][slot])
+            start, n = int(base["tileoffset"][g]) + (ci >> 16), ci & 0xFFFF
+            s16, codes = quantise_q4_ref(base["values"][start:start + n])
+            scales[slot] = s16
+            nibbles[start:start + n] = codes
+    codes = (nibbles[0::2] | (nibbles[1::2] << 4)).astype(np.uint8)
+    return dict(M=M, K=K, pad_elems=Q4_PAD, tileoffset=base["tileoffset"], colinfo=base["colinfo"],
+                bitmap=base["bitmap"], codes=codes, scales=scales, nnz=base["nnz"])
+
+
+def pack_q4_fast(W) -> dict:
+    """Same arrays as pack_q4_ref with whole-array NumPy steps (checked byte for byte against it)."""
+    Wb = as_bits(W)
+    base = pack_fast(Wb, pad_elems=Q4_PAD)
+    NGT = base["tileoffset"].shape[0] - 1
+    n = (base["colinfo"] & np.uint32(0xFFFF)).astype(np.int64)
+    start = np.repeat(base["tileoffset"][:-1].astype(np.int64), TILE_K) + (base["colinfo"] >> 16).astype(np.int64)
+    v32 = base["values"].view(np.float16).astype(np.float32)
+    owner = np.repeat(np.arange(NGT * TILE_K), pad_up(n, Q4_PAD))       # column tile of every (padded) element
+    stored = np.zeros(v32.shape[0], dtype=bool)
+    idx = np.concatenate([np.arange(s, s + k) for s, k in zip(start, n)]) if n.sum() else np.zeros(0, np.int64)
+    stored[idx] = True
+    mx = np.zeros(NGT * TILE_K, dtype=np.float32)
+    np.maximum.at(mx, owner[stored], np.abs(v32[stored]))
+    s16 = (mx / np.float32(7.0)).astype(np.float16)
+    s32 = s16.astype(np.float32)
+    per = s32[owner]
+    with np.errstate(divide="ignore", invalid="ignore"):
+        q = np.where(per == 0, np.float32(0), np.clip(np.rint(v32 / per), -7, 7))
+    nibbles = np.where(stored, q.astype(np.int32) + 8, 0).astype(np.uint8)
+    codes = (nibbles[0::2] | (nibbles[1::2] << 4)).astype(np.uint8)
+    return dict(M=base["M"], K=base["K"], pad_elems=Q4_PAD, tileoffset=base["tileoffset"], colinfo=base["colinfo"],
+                bitmap=base["bitmap"], codes=codes, scales=s16.view(np.uint16), nnz=base["nnz"])
+
+
+def dequant_q4_ref(p: dict) -> np.ndarray:
+    """The weights the 4-bit arrays stand for, dense float64 [M][K]: bit clear -> 0, else
+    (code - 8) * scale with the code found by the decode rule of Sec. 4.2.1 (rank = set bits before)."""
+    M, K = p["M"], p["K"]
+    R, C, _ = grid(M, K)
+    out = np.zeros((M, K), dtype=np.float64)
+    nib = np.empty(p["codes"].shape[0] * 2, dtype=np.uint8)
+    nib[0::2] = p["codes"] & 15
+    nib[1::2] = p["codes"] >> 4
+    for r in range(R):
+        for c in range(C):
+            g = r * C + c
+            for cc in range(TILE_K):
+                j = c * TILE_K + cc
+                slot = g * TILE_K + cc
+                nxt = int(p["tileoffset"][g]) + (int(p["colinfo"][slot]) >> 16)
+                s = float(np.uint16(p["scales"][slot]).view(np.float16))
+                for w in range(WORDS_PER_COL):
+                    word = int(p["bitmap"][slot * WORDS_PER_COL + w])
+                    for b in range(64):
+                        if (word >> b) & 1:
+                            out[r * TILE_M + 64 * w + b, j] = (int(nib[nxt]) - 8) * s
+                            nxt += 1
+    return out
+
+
+def spmspv_dense64_ref(Wd, x, active):
+    """The spMspV definition on a float64 weight matrix (the dequantised weights): (y, S)."""
+    xd = as_f64(x)
+    idx = np.flatnonzero(np.asarray(active, dtype=bool))
+    Wa = np.asarray(Wd, dtype=np.float64)[:, idx]
+    return Wa @ xd[idx], np.abs(Wa) @ np.abs(xd[idx])
+
+
+def active_bytes_q4(p: dict, active, y_bytes_per_elem: int = 2) -> int:
+    """Byte model of one call on the 4-bit variant: per active column tile 32 B of bitmap, its padded
+    codes (half a byte each), 4 B of ColInfo and 2 B of scale; TileOffset, x and y as before."""
+    M, K = p["M"], p["K"]
+    R, C, _ = grid(M, K)
+    a = np.zeros(C * TILE_K, dtype=bool)
+    a[:K] = np.asarray(active, dtype=bool)
+    n = (p["colinfo"] & np.uint32(0xFFFF)).astype(np.int64).reshape(R, C * TILE_K)
+    per_tile = 32 + pad_up(n, Q4_PAD) // 2 + 4 + 2
+    gt_active = int(a.reshape(C, TILE_K).any(axis=1).sum()) * R
+    return int(per_tile[:, a].sum()) + 4 * (gt_active + 1) + 2 * K + y_bytes_per_elem * M
+
+
 def tolerance(S) -> np.ndarray:
     """Per-output bound of the parity gate: 1e-3 * S[i] + 1e-5."""
     return 1e-3 * np.asarray(S, dtype=np.float64) + 1e-5

@@ -103,6 +103,29 @@ SPDP_API spdp_status spdp_pack_tiled_cbc(const void* W_dev, int64_t M, int64_t K
 SPDP_API spdp_status spdp_pack_tiled_cbc_ex(const void* W_dev, int64_t M, int64_t K, int64_t ldw,
                                    int tile_m, int tile_k, int pad_elems, void* stream, spdp_handle* out);
 
+/* Pack with a 4-bit Values payload (Sec. 5.1: 4-bit round-to-nearest weights, applied after static
+ * pruning and before dynamic pruning; Sec. 6: Values are stored apart from the sparsity metadata, so
+ * they can be low-bit).  The paper fixes no layout for it; this library's is: TileOffset, ColInfo and
+ * Bitmap exactly as in Sec. 4.1, with offsets counted in CODES and every column padded to 32 codes
+ * (16 bytes); Codes holds, per column tile, its n codes in row order, two per byte (even rank in the
+ * low nibble), zero padded; Scales holds one fp16 per column tile (same index as ColInfo).
+ *   scale = fp16(max|w| of the column tile / 7), computed in fp32;
+ *   code  = clamp(rint(w / scale), -7, 7) + 8 in fp32, ties to even (8 where the scale is 0);
+ *   the weight a code stands for is (code - 8) * scale.
+ * Weights must be finite (codes of Inf/NaN are unspecified).  Arguments as spdp_pack_tiled_cbc.
+ * The handle works with spdp_spmspv, spdp_spmspv_host, spdp_active_columns, spdp_get_info
+ * (pad_elems = 32, values_len = number of codes), spdp_set_num_ctas and spdp_export_q4; the other
+ * calls return SPDP_ERR_UNSUPPORTED_SHAPE for it.  spdp_spmspv on such a handle computes
+ * y = sum over active columns of (code - 8) * scale * x_j with fp32 accumulation. */
+SPDP_API spdp_status spdp_pack_tiled_cbc_q4(const void* W_dev, int64_t M, int64_t K, int64_t ldw, int tile_m,
+                                   int tile_k, void* stream, spdp_handle* out);
+
+/* Copy the arrays of a 4-bit handle to HOST buffers: tileoffset uint32[NGT+1], colinfo uint32[NGT*16],
+ * bitmap uint64[NGT*64], codes uint8[values_len/2], scales fp16[NGT*16] (any pointer may be NULL).
+ * Synchronous.  SPDP_ERR_INVALID_ARG for a handle that is not 4-bit. */
+SPDP_API spdp_status spdp_export_q4(spdp_handle h, void* tileoffset_host, void* colinfo_host, void* bitmap_host,
+                           void* codes_host, void* scales_host);
+
 /* Build a handle from the four Tiled-CBC arrays in HOST memory (Sec. 4.1).  The arrays are
  * validated on the host (monotone TileOffset, ColInfo offsets equal to the prefix sums of the
  * padded counts, bitmap popcounts equal to the ColInfo counts); a mismatch returns

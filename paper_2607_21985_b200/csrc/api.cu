@@ -25,6 +25,7 @@ void release(spdp_matrix* h) {
     cudaFree(h->colinfo);
     cudaFree(h->bitmap);
     cudaFree(h->values);
+    cudaFree(h->scales);
     cudaFree(h->workspace);
     cudaFree(h->workspace_batch);
     cudaFree(h->status_word);
@@ -41,7 +42,7 @@ void release(spdp_matrix* h) {
 
 spdp_status new_handle(int64_t M, int64_t K, int pad_elems, spdp_matrix** out) {
     if (M < 1 || K < 1 || M > (int64_t(1) << 30) || K > (int64_t(1) << 30)) return SPDP_ERR_UNSUPPORTED_SHAPE;
-    if (pad_elems != 8 && pad_elems != 1) return SPDP_ERR_UNSUPPORTED_SHAPE;
+    if (pad_elems != 8 && pad_elems != 1 && pad_elems != 32) return SPDP_ERR_UNSUPPORTED_SHAPE;
     spdp_matrix* h = new (std::nothrow) spdp_matrix();
     if (h == nullptr) return SPDP_ERR_ALLOC;
     std::memset(h, 0, sizeof(*h));
@@ -109,6 +110,12 @@ spdp_status finish_handle(spdp_matrix* h) {
 
 constexpr int kBatchViaSingleCalls = 2;   // spdp_spmspv_batch: up to this many tokens go through the single-vector kernel
 
+// The decode kernel of the handle's Values variant (fp16 values, or 4-bit codes with scales).
+spdp_status launch_decode(const spdp_matrix* h, const __half* x, int rule, float thr, const uint32_t* mask, void* y,
+                          int ydt, cudaStream_t s) {
+    return h->q4 ? launch_spmspv_q4(h, x, rule, thr, mask, y, ydt, s) : launch_spmspv(h, x, rule, thr, mask, y, ydt, s);
+}
+
 bool rule_ok(int rule) { return rule == SPDP_DP_NONE || rule == SPDP_DP_ABS_GT || rule == SPDP_DP_MASK; }
 
 }  // namespace
@@ -126,7 +133,7 @@ spdp_status enqueue_host_call(spdp_matrix* h, const void* x_host, int rule, floa
     if (rule == SPDP_DP_MASK)
         SPDP_CUDA_TRY(cudaMemcpyAsync(h->mask_stage, mask_host, ((h->K + 31) / 32) * sizeof(uint32_t),
                                       cudaMemcpyHostToDevice, s));
-    spdp_status st = launch_spmspv(h, h->x_stage, rule, thr, rule == SPDP_DP_MASK ? h->mask_stage : nullptr,
+    spdp_status st = launch_decode(h, h->x_stage, rule, thr, rule == SPDP_DP_MASK ? h->mask_stage : nullptr,
                                    h->y_stage, ydt, s);
     if (st != SPDP_OK) return st;
     const size_t ybytes = static_cast<size_t>(h->M) * (ydt == SPDP_Y_F32 ? sizeof(float) : sizeof(__half));
@@ -188,6 +195,7 @@ spdp_status spdp_pack_tiled_cbc_ex(const void* W_dev, int64_t M, int64_t K, int6
     if (W_dev == nullptr || out == nullptr) return SPDP_ERR_INVALID_ARG;
     if (tile_m != kTileM || tile_k != kTileK) return SPDP_ERR_UNSUPPORTED_SHAPE;
     if (M < 1 || K < 1 || ldw < K) return SPDP_ERR_UNSUPPORTED_SHAPE;
+    if (pad_elems != 8 && pad_elems != 1) return SPDP_ERR_UNSUPPORTED_SHAPE;
     if (reinterpret_cast<uintptr_t>(W_dev) & 1u) return SPDP_ERR_INVALID_ARG;
     spdp_matrix* h = nullptr;
     spdp_status st = new_handle(M, K, pad_elems, &h);
@@ -202,6 +210,41 @@ spdp_status spdp_pack_tiled_cbc_ex(const void* W_dev, int64_t M, int64_t K, int6
 spdp_status spdp_pack_tiled_cbc(const void* W_dev, int64_t M, int64_t K, int64_t ldw, int tile_m,
                                 int tile_k, void* stream, spdp_handle* out) {
     return spdp_pack_tiled_cbc_ex(W_dev, M, K, ldw, tile_m, tile_k, 8, stream, out);
+}
+
+spdp_status spdp_pack_tiled_cbc_q4(const void* W_dev, int64_t M, int64_t K, int64_t ldw, int tile_m, int tile_k,
+                                   void* stream, spdp_handle* out) {
+    if (W_dev == nullptr || out == nullptr) return SPDP_ERR_INVALID_ARG;
+    if (tile_m != kTileM || tile_k != kTileK) return SPDP_ERR_UNSUPPORTED_SHAPE;
+    if (M < 1 || K < 1 || ldw < K) return SPDP_ERR_UNSUPPORTED_SHAPE;
+    if (reinterpret_cast<uintptr_t>(W_dev) & 1u) return SPDP_ERR_INVALID_ARG;
+    spdp_matrix* h = nullptr;
+    spdp_status st = new_handle(M, K, 32, &h);
+    if (st != SPDP_OK) return st;
+    h->q4 = 1;
+    st = pack_q4_device(h, static_cast<const __half*>(W_dev), ldw, static_cast<cudaStream_t>(stream));
+    if (st == SPDP_OK) st = finish_handle(h);
+    if (st != SPDP_OK) { release(h); return st; }
+    *out = h;
+    return SPDP_OK;
+}
+
+spdp_status spdp_export_q4(spdp_handle h, void* tileoffset_host, void* colinfo_host, void* bitmap_host, void* codes_host,
+                           void* scales_host) {
+    if (!valid(h) || !h->q4) return SPDP_ERR_INVALID_ARG;
+    SPDP_CUDA_TRY(cudaDeviceSynchronize());
+    if (tileoffset_host)
+        SPDP_CUDA_TRY(cudaMemcpy(tileoffset_host, h->tileoffset, (h->NGT + 1) * sizeof(uint32_t), cudaMemcpyDeviceToHost));
+    if (colinfo_host)
+        SPDP_CUDA_TRY(cudaMemcpy(colinfo_host, h->colinfo, h->NGT * kTileK * sizeof(uint32_t), cudaMemcpyDeviceToHost));
+    if (bitmap_host)
+        SPDP_CUDA_TRY(cudaMemcpy(bitmap_host, h->bitmap, h->NGT * kTileK * kWordsPerCol * sizeof(uint64_t),
+                                 cudaMemcpyDeviceToHost));
+    if (codes_host && h->values_len > 0)
+        SPDP_CUDA_TRY(cudaMemcpy(codes_host, h->values, h->values_len / 2, cudaMemcpyDeviceToHost));
+    if (scales_host)
+        SPDP_CUDA_TRY(cudaMemcpy(scales_host, h->scales, h->NGT * kTileK * sizeof(__half), cudaMemcpyDeviceToHost));
+    return SPDP_OK;
 }
 
 spdp_status spdp_import_tiled_cbc(int64_t M, int64_t K, int pad_elems, const void* tileoffset_host,
@@ -265,10 +308,10 @@ spdp_status spdp_spmspv(spdp_handle h, const void* x_dev, spdp_dp_rule rule, flo
         (reinterpret_cast<uintptr_t>(y_dev) & (ydt == SPDP_Y_F32 ? 3u : 1u)) ||
         (reinterpret_cast<uintptr_t>(mask_dev) & 3u))
         return SPDP_ERR_INVALID_ARG;
-    if (h->pad_elems != 8) return SPDP_ERR_UNSUPPORTED_SHAPE;
+    if (h->pad_elems != 8 && !h->q4) return SPDP_ERR_UNSUPPORTED_SHAPE;
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev != h->device) return SPDP_ERR_INVALID_ARG;   // wrong current device
-    return launch_spmspv(h, static_cast<const __half*>(x_dev), rule, thr,
+    return launch_decode(h, static_cast<const __half*>(x_dev), rule, thr,
                          static_cast<const uint32_t*>(mask_dev), y_dev, ydt, static_cast<cudaStream_t>(stream));
 }
 
@@ -344,7 +387,7 @@ spdp_status spdp_spmspv_host(spdp_handle h, const void* x_host, spdp_dp_rule rul
     if (!valid(h) || x_host == nullptr || y_host == nullptr) return SPDP_ERR_INVALID_ARG;
     if (!rule_ok(rule) || (ydt != SPDP_Y_F16 && ydt != SPDP_Y_F32)) return SPDP_ERR_INVALID_ARG;
     if (rule == SPDP_DP_MASK && mask_host == nullptr) return SPDP_ERR_INVALID_ARG;
-    if (h->pad_elems != 8) return SPDP_ERR_UNSUPPORTED_SHAPE;
+    if (h->pad_elems != 8 && !h->q4) return SPDP_ERR_UNSUPPORTED_SHAPE;
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev != h->device) return SPDP_ERR_INVALID_ARG;   // wrong current device
     cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -392,7 +435,8 @@ spdp_status spdp_get_info(spdp_handle h, spdp_info* out) {
     i.pad_elems = h->pad_elems;
     i.nnz = h->nnz;
     i.values_len = h->values_len;
-    i.packed_bytes = (h->NGT + 1) * 4 + h->NGT * kTileK * 4 + h->NGT * kTileK * kWordsPerCol * 8 + h->values_len * 2;
+    i.packed_bytes = (h->NGT + 1) * 4 + h->NGT * kTileK * 4 + h->NGT * kTileK * kWordsPerCol * 8 +
+                     (h->q4 ? h->values_len / 2 + h->NGT * kTileK * 2 : h->values_len * 2);
     i.workspace_bytes = h->workspace_bytes;
     i.tileoffset_dev = h->tileoffset;
     i.colinfo_dev = h->colinfo;
@@ -407,6 +451,7 @@ spdp_status spdp_get_info(spdp_handle h, spdp_info* out) {
 spdp_status spdp_export(spdp_handle h, void* tileoffset_host, void* colinfo_host, void* bitmap_host,
                         void* values_host) {
     if (!valid(h)) return SPDP_ERR_INVALID_ARG;
+    if (h->q4) return SPDP_ERR_UNSUPPORTED_SHAPE;           // 4-bit handles: spdp_export_q4
     SPDP_CUDA_TRY(cudaDeviceSynchronize());
     if (tileoffset_host)
         SPDP_CUDA_TRY(cudaMemcpy(tileoffset_host, h->tileoffset, (h->NGT + 1) * sizeof(uint32_t), cudaMemcpyDeviceToHost));
@@ -422,7 +467,7 @@ spdp_status spdp_export(spdp_handle h, void* tileoffset_host, void* colinfo_host
 
 spdp_status spdp_unpack(spdp_handle h, void* W_dev_out, int64_t ldw, void* stream) {
     if (!valid(h) || W_dev_out == nullptr) return SPDP_ERR_INVALID_ARG;
-    if (ldw < h->K) return SPDP_ERR_UNSUPPORTED_SHAPE;
+    if (ldw < h->K || h->q4) return SPDP_ERR_UNSUPPORTED_SHAPE;
     return unpack_device(h, static_cast<__half*>(W_dev_out), ldw, static_cast<cudaStream_t>(stream));
 }
 

@@ -135,6 +135,67 @@ pack_emit_kernel(const unsigned short* __restrict__ W, int64_t ldw, int64_t M, i
     }
 }
 
+// Pass 3 of the 4-bit variant (Sec. 5.1, 4-bit round to nearest, after static pruning): one fp16 scale
+// per column tile = max|w| / 7, code = clamp(rint(w / scale), -7, 7) + 8 in fp32 (ties to even; code 8
+// where the scale underflows to 0), the column's codes in row order, two per byte, low nibble first.
+__global__ void __launch_bounds__(kTileM)
+pack_q4_emit_kernel(const unsigned short* __restrict__ W, int64_t ldw, int64_t M, int64_t K, int64_t C,
+                    const uint32_t* __restrict__ tileoffset, const uint32_t* __restrict__ colinfo,
+                    unsigned char* __restrict__ codes, unsigned short* __restrict__ scales) {
+    __shared__ unsigned words32[kTileK][kTileM / 32];
+    __shared__ float warp_max[kTileK][kTileM / 32];
+    __shared__ unsigned char by_rank[kTileK][kTileM];
+    const int64_t g = blockIdx.x;
+    const int64_t r = g / C, c = g % C;
+    const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+    unsigned short v[kTileK];
+    load_tile_row(W, ldw, M, K, r * kTileM + t, c * kTileK, v);
+    unsigned mine[kTileK];
+#pragma unroll
+    for (int cc = 0; cc < kTileK; ++cc) {
+        mine[cc] = __ballot_sync(0xFFFFFFFFu, is_stored(v[cc]));
+        float a = is_stored(v[cc]) ? fabsf(__half2float(__ushort_as_half(v[cc]))) : 0.f;
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) a = fmaxf(a, __shfl_xor_sync(0xFFFFFFFFu, a, d));
+        if (lane == 0) {
+            words32[cc][warp] = mine[cc];
+            warp_max[cc][warp] = a;
+        }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int cc = 0; cc < kTileK; ++cc) {
+        float mx = 0.f;
+#pragma unroll
+        for (int w = 0; w < kTileM / 32; ++w) mx = fmaxf(mx, warp_max[cc][w]);
+        const __half s16 = __float2half_rn(__fdiv_rn(mx, 7.0f));
+        if (t == 0) scales[g * kTileK + cc] = __half_as_ushort(s16);
+        if (!is_stored(v[cc])) continue;
+        const float sf = __half2float(s16);
+        int q = 0;
+        if (sf != 0.f) {
+            q = static_cast<int>(rintf(__fdiv_rn(__half2float(__ushort_as_half(v[cc])), sf)));
+            q = q < -7 ? -7 : (q > 7 ? 7 : q);
+        }
+        unsigned rank = __popc(mine[cc] & ((1u << lane) - 1u));
+        for (int w = 0; w < warp; ++w) rank += __popc(words32[cc][w]);
+        by_rank[cc][rank] = static_cast<unsigned char>(q + 8);
+    }
+    __syncthreads();
+    const uint64_t base = tileoffset[g];
+    if (t < kTileM / 2) {
+#pragma unroll
+        for (int cc = 0; cc < kTileK; ++cc) {
+            const uint32_t ci = colinfo[g * kTileK + cc];
+            const int n = static_cast<int>(ci & 0xFFFFu);
+            if (2 * t < n) {
+                const unsigned lo = by_rank[cc][2 * t], hi = (2 * t + 1 < n) ? by_rank[cc][2 * t + 1] : 0u;
+                codes[((base + (ci >> 16)) >> 1) + t] = static_cast<unsigned char>(lo | (hi << 4));
+            }
+        }
+    }
+}
+
 // Decode rule of Sec. 4.2.1: bit clear -> +0, else Values[base + set bits before the position].
 __global__ void __launch_bounds__(kTileM)
 unpack_kernel(const uint32_t* __restrict__ tileoffset, const uint32_t* __restrict__ colinfo,
@@ -201,6 +262,50 @@ spdp_status pack_device(spdp_matrix* h, const __half* W, int64_t ldw, cudaStream
         e = cudaStreamSynchronize(s);
         if (e == cudaSuccess) e = cudaGetLastError();
         if (e != cudaSuccess) { note_cuda_error(e, "pack emit"); st = SPDP_ERR_CUDA; break; }
+    } while (false);
+    cudaFree(tile_len);
+    cudaFree(total_dev);
+    return st;
+}
+
+// The 4-bit variant: same count and scan passes with a padding unit of 32 codes, then the quantising emit.
+spdp_status pack_q4_device(spdp_matrix* h, const __half* W, int64_t ldw, cudaStream_t s) {
+    const int64_t NGT = h->NGT;
+    uint32_t* tile_len = nullptr;
+    unsigned long long* total_dev = nullptr;
+    SPDP_CUDA_TRY(cudaMalloc(&h->tileoffset, (NGT + 1) * sizeof(uint32_t)));
+    SPDP_CUDA_TRY(cudaMalloc(&h->colinfo, NGT * kTileK * sizeof(uint32_t)));
+    SPDP_CUDA_TRY(cudaMalloc(&h->bitmap, NGT * kTileK * kWordsPerCol * sizeof(uint64_t)));
+    SPDP_CUDA_TRY(cudaMalloc(&h->scales, NGT * kTileK * sizeof(__half)));
+    SPDP_CUDA_TRY(cudaMalloc(&tile_len, NGT * sizeof(uint32_t)));
+    cudaError_t e = cudaMalloc(&total_dev, 2 * sizeof(unsigned long long));   // [0] code count, [1] nnz
+    if (e != cudaSuccess) { cudaFree(tile_len); SPDP_CUDA_TRY(e); }
+    const unsigned short* Wb = reinterpret_cast<const unsigned short*>(W);
+    spdp_status st = SPDP_OK;
+    unsigned long long totals[2] = {0, 0};
+    do {
+        e = cudaMemsetAsync(total_dev, 0, 2 * sizeof(unsigned long long), s);
+        if (e != cudaSuccess) { note_cuda_error(e, "cudaMemsetAsync(totals)"); st = SPDP_ERR_CUDA; break; }
+        pack_count_kernel<<<static_cast<unsigned>(NGT), kTileM, 0, s>>>(
+            Wb, ldw, h->M, h->K, h->C, h->pad_elems, h->bitmap, h->colinfo, tile_len, total_dev + 1);
+        pack_scan_kernel<<<1, 1024, 0, s>>>(tile_len, NGT, h->tileoffset, total_dev);
+        e = cudaMemcpyAsync(totals, total_dev, sizeof(totals), cudaMemcpyDeviceToHost, s);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+        if (e != cudaSuccess) { note_cuda_error(e, "pack count/scan"); st = SPDP_ERR_CUDA; break; }
+        if (totals[0] >= (1ull << 32)) { st = SPDP_ERR_OVERFLOW; break; }
+        h->values_len = static_cast<int64_t>(totals[0]);
+        h->nnz = static_cast<int64_t>(totals[1]);
+        const size_t cbytes = static_cast<size_t>(totals[0]) / 2 + 16;         // + 16: the decode reads one word past a span
+        e = cudaMalloc(&h->values, cbytes);
+        if (e != cudaSuccess) { note_cuda_error(e, "cudaMalloc(codes)"); st = SPDP_ERR_ALLOC; break; }
+        e = cudaMemsetAsync(h->values, 0, cbytes, s);
+        if (e != cudaSuccess) { note_cuda_error(e, "cudaMemsetAsync(codes)"); st = SPDP_ERR_CUDA; break; }
+        pack_q4_emit_kernel<<<static_cast<unsigned>(NGT), kTileM, 0, s>>>(
+            Wb, ldw, h->M, h->K, h->C, h->tileoffset, h->colinfo, reinterpret_cast<unsigned char*>(h->values),
+            reinterpret_cast<unsigned short*>(h->scales));
+        e = cudaStreamSynchronize(s);
+        if (e == cudaSuccess) e = cudaGetLastError();
+        if (e != cudaSuccess) { note_cuda_error(e, "pack q4 emit"); st = SPDP_ERR_CUDA; break; }
     } while (false);
     cudaFree(tile_len);
     cudaFree(total_dev);

@@ -100,7 +100,7 @@ __global__ void probe_gather_kernel(const uint2* __restrict__ items, const unsig
 }  // namespace
 
 spdp_status launch_probe_stream_read(const spdp_matrix* h, cudaStream_t s) {
-    const long long n16 = h->values_len * 2 / 16;
+    const long long n16 = (h->q4 ? h->values_len / 2 : h->values_len * 2) / 16;      // bytes of the Values payload / 16
     probe_stream_read_kernel<<<h->sm_count * 8, 256, 0, s>>>(reinterpret_cast<const uint4*>(h->values), n16,
                                                              reinterpret_cast<unsigned*>(h->status_word) + 1);
     SPDP_CUDA_TRY(cudaGetLastError());

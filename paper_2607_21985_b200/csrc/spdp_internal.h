@@ -30,7 +30,9 @@ struct spdp_matrix {
     uint32_t* tileoffset;   // [NGT+1]
     uint32_t* colinfo;      // [NGT*16]
     uint64_t* bitmap;       // [NGT*16*4]
-    __half* values;         // [values_len] (at least 16 bytes are allocated)
+    __half* values;         // [values_len] (at least 16 bytes are allocated); 4-bit variant: values_len codes, two per byte
+    int q4;                 // 1: the 4-bit variant (codes + scales), pad_elems = 32
+    __half* scales;         // 4-bit variant: [NGT*16] one scale per column tile; else null
 
     // Work partition of one spmspv launch: the kernel cuts the NGT GTiles into num_ctas equal
     // contiguous ranges, one per CTA.
@@ -106,6 +108,11 @@ spdp_status configure_spmspv_batch_kernel();   // per-device kernel attributes; 
 spdp_status launch_spmspv_batch(const spdp_matrix* h, const __half* x, int64_t ldx, int batch, int rule, float thr,
                                 const uint32_t* mask, int64_t mask_stride, void* y, int64_t ldy, int ydt,
                                 cudaStream_t s);
+
+// spmspv_q4.cu / pack.cu: the 4-bit variant
+spdp_status pack_q4_device(spdp_matrix* h, const __half* W, int64_t ldw, cudaStream_t s);
+spdp_status launch_spmspv_q4(const spdp_matrix* h, const __half* x, int rule, float thr, const uint32_t* mask, void* y,
+                             int ydt, cudaStream_t s);
 
 // spmm.cu
 spdp_status configure_spmm_kernel();            // per-device kernel attributes; idempotent

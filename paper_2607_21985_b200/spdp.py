@@ -29,7 +29,7 @@ EXPORTS = (
     "spdp_pack_tiled_cbc", "spdp_pack_tiled_cbc_ex", "spdp_import_tiled_cbc", "spdp_spmspv",
     "spdp_spmspv_host", "spdp_spmspv_noalloc", "spdp_spmspv_batch", "spdp_free", "spdp_get_info", "spdp_export", "spdp_unpack",
     "spdp_active_columns", "spdp_last_device_status", "spdp_set_num_ctas", "spdp_last_cuda_error",
-    "spdp_status_string", "spdp_probe_stream_read", "spdp_probe_gather", "spdp_spmm",
+    "spdp_status_string", "spdp_probe_stream_read", "spdp_probe_gather", "spdp_spmm", "spdp_pack_tiled_cbc_q4", "spdp_export_q4",
 )
 
 
@@ -75,6 +75,8 @@ def lib():
         L.spdp_last_device_status.argtypes = [vp, ctypes.POINTER(ci)]
         L.spdp_set_num_ctas.argtypes = [vp, ci]
         L.spdp_spmm.argtypes = [vp, vp, i64, i64, vp, i64, ci, vp]
+        L.spdp_pack_tiled_cbc_q4.argtypes = [vp, i64, i64, i64, ci, ci, vp, ctypes.POINTER(vp)]
+        L.spdp_export_q4.argtypes = [vp, vp, vp, vp, vp, vp]
         L.spdp_probe_stream_read.argtypes = [vp, vp]
         L.spdp_probe_gather.argtypes = [vp, vp, ci, cf, vp, vp]
         for name in EXPORTS:
@@ -138,6 +140,33 @@ def spdp_pack_tiled_cbc(W, tile_m: int = 256, tile_k: int = 16, stream=None, pad
                                           _stream(stream), ctypes.byref(h))
     _check(st, "spdp_pack_tiled_cbc")
     return h.value
+
+
+def spdp_pack_tiled_cbc_q4(W, stream=None) -> int:
+    """W: fp16 CUDA tensor [M, K] -> handle of the 4-bit variant (codes + one fp16 scale per column tile)."""
+    import torch
+    if W.dtype != torch.float16 or W.dim() != 2 or not W.is_cuda or W.stride(1) != 1:
+        raise ValueError("W must be a 2-D fp16 CUDA tensor with unit column stride")
+    M, K = W.shape
+    h = ctypes.c_void_p()
+    st = lib().spdp_pack_tiled_cbc_q4(W.data_ptr(), M, K, W.stride(0), 256, 16, _stream(stream), ctypes.byref(h))
+    _check(st, "spdp_pack_tiled_cbc_q4")
+    return h.value
+
+
+def spdp_export_q4(h: int) -> dict:
+    """The arrays of a 4-bit handle as NumPy arrays (synchronous device-to-host copies)."""
+    info = spdp_get_info(h)
+    to = np.empty(info.NGT + 1, np.uint32)
+    ci = np.empty(info.NGT * 16, np.uint32)
+    bm = np.empty(info.NGT * 64, np.uint64)
+    codes = np.empty(info.values_len // 2, np.uint8)
+    scales = np.empty(info.NGT * 16, np.uint16)
+    st = lib().spdp_export_q4(h, to.ctypes.data, ci.ctypes.data, bm.ctypes.data, codes.ctypes.data if codes.size else None,
+                              scales.ctypes.data)
+    _check(st, "spdp_export_q4")
+    return dict(M=info.M, K=info.K, pad_elems=info.pad_elems, tileoffset=to, colinfo=ci, bitmap=bm, codes=codes,
+                scales=scales, nnz=info.nnz)
 
 
 def spdp_import_tiled_cbc(M: int, K: int, tileoffset, colinfo, bitmap, values, pad_elems: int = 8) -> int:

@@ -392,6 +392,152 @@ def run_prefill(args):
     spdp.spdp_free(h)
 
 
+def run_q4(args):
+    """--q4: the decode call on the 4-bit Values variant of the same layer (Sec. 5.1 / Sec. 6).  A side
+    measurement: the byte model shrinks to half a byte per stored weight plus one fp16 scale per column tile."""
+    import torch
+    from oracle import spdp_oracle as O
+    from paper_2607_21985_b200 import spdp
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    spdp.lib()
+    w = make_workload(args.workload)
+    l2 = torch.cuda.get_device_properties(0).L2_cache_size
+    Wd = torch.from_numpy(w.W).cuda()
+    h0 = spdp.spdp_pack_tiled_cbc_q4(Wd)
+    info = spdp.spdp_get_info(h0)
+    packed = spdp.spdp_export_q4(h0)
+    a = O.active_ref(w.x, w.rule, w.thr)
+    B_active = O.active_bytes_q4(packed, a, 2)           # the oracle's byte model on the exported arrays
+    copies = args.copies or max(2, int(np.ceil(2 * l2 / B_active)) + 1)
+    handles = [h0] + [spdp.spdp_pack_tiled_cbc_q4(Wd) for _ in range(copies - 1)]
+    xs = [torch.from_numpy(w.x).cuda() for _ in range(copies)]
+    ys = [torch.empty(w.M, dtype=torch.float16, device="cuda") for _ in range(copies)]
+    for i in range(args.warmup):
+        spdp.spdp_spmspv(handles[i % copies], xs[i % copies], w.rule, w.thr, ys[i % copies])
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        spdp.spdp_spmspv(handles[i % copies], xs[i % copies], w.rule, w.thr, ys[i % copies])
+    e1.record()
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) / args.steps * 1e3
+    assert all(spdp.spdp_last_device_status(h) == 0 for h in handles)
+    # parity on the rows of three row tiles, against the oracle's product on the dequantised weights
+    yh = ys[0].float().cpu().numpy().astype(np.float64)
+    worst = 0.0
+    R = (w.M + 255) // 256
+    for r in sorted(set([0, R // 2, R - 1])):
+        sub = O.pack_q4_fast(w.W[256 * r:256 * (r + 1)])
+        y_ref, S = O.spmspv_dense64_ref(O.dequant_q4_ref(sub), w.x, a)
+        worst = max(worst, float(np.max(np.abs(yh[256 * r:256 * r + y_ref.shape[0]] - y_ref) / (1e-3 * S + 1e-5))))
+    assert worst <= 1.0, "4-bit result outside 1e-3 * S + 1e-5 of the dequantised product"
+    peak, peak_kind = measured_peak()
+    achieved = B_active / (us * 1e-6) / 1e9
+    print(json.dumps({
+        "metric": "spmspv_q4_effective_hbm_gbs", "value": achieved, "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": us * 1e-3, "us_per_call": us, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "storage": "4-bit codes + fp16 scale per column tile", "active_bytes_per_call": int(B_active),
+                   "packed_bytes": int(info.packed_bytes), "copies": copies,
+                   "l2": "inputs larger than L2: rotating packed copies"},
+        "gpu_launches": args.steps,
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "peak_kind": f"of {peak_kind}", "traffic": None, "kernel": "spmspv_q4_kernel",
+                     "algorithmic_bytes": int(B_active)},
+        "parity": {"max_normalised_error_sampled_row_tiles": worst},
+    }))
+    for h in handles:
+        spdp.spdp_free(h)
+
+
+def run_sharded(args):
+    """--sharded: ONE layer split by row tiles over the N ranks (strong scaling): every rank packs its rows,
+    runs the decode call on the replicated x and joins the slices of y with one NCCL all-gather."""
+    import torch
+    import torch.distributed as dist
+    from paper_2607_21985_b200 import spdp
+    from paper_2607_21985_b200.sharded import RowShardedMatrix
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    spdp.lib()
+    w = make_workload(args.workload)
+    l2 = torch.cuda.get_device_properties(local).L2_cache_size
+    first, rows = spdp.spdp_row_shard(w.M, world, rank)
+    packs = []
+
+    def pack(rows_of_w):
+        h = spdp.spdp_pack_tiled_cbc(torch.from_numpy(np.ascontiguousarray(rows_of_w)).cuda())
+        packs.append(h)
+        return h
+
+    # algorithmic bytes: of the whole layer (the value's numerator) and of this rank's share (for the copies)
+    h_probe = pack(w.W[first:first + rows])
+    words = torch.zeros((w.K + 31) // 32, dtype=torch.int32, device="cuda")
+    spdp.spdp_active_columns(h_probe, torch.from_numpy(w.x).cuda(), w.rule, w.thr, words)
+    torch.cuda.synchronize()
+    aw = words.cpu().numpy().view(np.uint32)
+    B_local = active_bytes(spdp.spdp_export(h_probe)["colinfo"], aw, rows, w.K, 2)
+    copies = args.copies or max(2, int(np.ceil(2 * l2 / B_local)) + 1)
+    shards = [RowShardedMatrix(w.M, w.K, lambda r0, n: w.W[r0:r0 + n], pack,
+                               lambda h, x, ys: spdp.spdp_spmspv(h, x, w.rule, w.thr, ys), device="cuda")
+              for _ in range(copies)]
+    xs = [torch.from_numpy(w.x).cuda() for _ in range(copies)]
+    t_bytes = torch.tensor([float(B_local - 2 * w.K)], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t_bytes)
+    B_total = float(t_bytes.item()) + 2 * w.K          # every rank reads x; counted once, as in the one-GPU model
+
+    def step(i):
+        return shards[i % copies].spmspv(xs[i % copies])
+
+    for i in range(args.warmup):
+        step(i)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        y = step(i)
+    e1.record()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    ms = max_over_ranks(e0.elapsed_time(e1), world) / args.steps
+    if rank == 0:
+        from oracle import c_oracle
+        a = c_oracle.active(w.x, w.rule, w.thr)
+        rows_chk = min(w.M, 2048)
+        y_ref, S, _ = c_oracle.spmspv(w.W[:rows_chk], w.x, a, want_scale=True)
+        err = np.abs(y[:rows_chk].float().cpu().numpy().astype(np.float64) - y_ref) / (1e-3 * S + 1e-5)
+        assert float(err.max()) <= 1.0, "sharded result outside 1e-3 * S + 1e-5"
+        peak, peak_kind = measured_peak()
+        value = B_total / (ms * 1e-3) / 1e9
+        print(json.dumps({
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms, "us_per_call": ms * 1e3, "higher_is_better": True, "scaling": "strong", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": w.name, "parallelism": f"row tiles over {world} ranks + all-gather of y",
+                       "rows_rank0": rows, "active_bytes_per_call": int(B_total), "copies": copies,
+                       "l2": "inputs larger than L2: rotating packed copies per rank"},
+            "gpu_launches": args.steps,
+            "roofline": {"bound": "hbm", "achieved": value / world, "peak": peak, "unit": "GB/s", "frac": value / world / peak,
+                         "peak_kind": f"of {peak_kind}, per GPU", "traffic": None, "kernel": "spmspv_kernel",
+                         "algorithmic_bytes": int(B_total)},
+            "parity": {"max_normalised_error_first_rows": float(err.max())},
+        }))
+    for h in packs:
+        spdp.spdp_free(h)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -405,6 +551,9 @@ def main():
     ap.add_argument("--no-context", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay timing")
     ap.add_argument("--batch", type=int, default=1, help="2..8: time the small-batch entry point instead (1 GPU)")
+    ap.add_argument("--sharded", action="store_true",
+                    help="split ONE layer by row tiles over the ranks and all-gather y (strong scaling) instead of replicas")
+    ap.add_argument("--q4", action="store_true", help="time the decode call on the 4-bit Values variant instead (1 GPU)")
     ap.add_argument("--prefill", type=int, default=0, help="N > 0: time the prefill entry point with N tokens instead (1 GPU)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
@@ -417,6 +566,12 @@ def main():
         return
     if args.prefill > 0:
         run_prefill(args)
+        return
+    if args.q4:
+        run_q4(args)
+        return
+    if args.sharded:
+        run_sharded(args)
         return
 
     import torch

@@ -220,6 +220,14 @@ SPDP_API spdp_status spdp_spmspv_noalloc(const void* tileoffset_dev, const void*
                                 const void* x_dev, spdp_dp_rule rule, float thr, const void* mask_dev,
                                 void* y_dev, spdp_ydtype ydt, void* stream);
 
+/* Row-tile sharding over several GPUs (the paper names multi-GPU execution as future work, Sec. 6; the
+ * natural split of y = W x keeps whole 256-row tiles together, so every rank packs its own rows as
+ * an independent Tiled-CBC matrix, x is replicated, and the outputs are disjoint).  This is the split
+ * every rank must agree on: the ceil(M/256) row tiles are dealt out in contiguous runs, the first
+ * (tiles % world) ranks get one more.  Writes rank's first row and its number of rows (0 when there
+ * are fewer row tiles than ranks).  Host arithmetic only. */
+SPDP_API spdp_status spdp_row_shard(int64_t M, int world, int rank, int64_t* first_row_out, int64_t* rows_out);
+
 /* Release the handle and everything it owns.  spdp_free(NULL) is SPDP_OK. */
 SPDP_API spdp_status spdp_free(spdp_handle h);
 

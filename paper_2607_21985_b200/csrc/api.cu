@@ -420,6 +420,21 @@ spdp_status spdp_spmspv_host(spdp_handle h, const void* x_host, spdp_dp_rule rul
     return SPDP_OK;
 }
 
+spdp_status spdp_row_shard(int64_t M, int world, int rank, int64_t* first_row_out, int64_t* rows_out) {
+    if (M < 1 || world < 1 || rank < 0 || rank >= world || first_row_out == nullptr || rows_out == nullptr)
+        return SPDP_ERR_INVALID_ARG;
+    const int64_t tiles = (M + kTileM - 1) / kTileM;
+    const int64_t base = tiles / world, extra = tiles % world;
+    const int64_t first_tile = rank * base + (rank < extra ? rank : extra);
+    const int64_t my_tiles = base + (rank < extra ? 1 : 0);
+    const int64_t first = first_tile * kTileM;
+    int64_t last = (first_tile + my_tiles) * kTileM;
+    if (last > M) last = M;
+    *first_row_out = first < M ? first : M;
+    *rows_out = last > first ? last - first : 0;
+    return SPDP_OK;
+}
+
 spdp_status spdp_free(spdp_handle h) {
     if (h == nullptr) return SPDP_OK;
     if (!valid(h)) return SPDP_ERR_INVALID_ARG;

@@ -79,40 +79,60 @@ spmspv_q4_kernel(const __grid_constant__ QParams p) {
                     sx = __half2float(__ldg(p.scales + g * kTileK + lane)) * __half2float(xj);   // exact in fp32
                 }
             }
-            unsigned am = __ballot_sync(0xFFFFFFFFu, act) & 0xFFFFu;
+            const unsigned am = __ballot_sync(0xFFFFFFFFu, act) & 0xFFFFu;
             const unsigned to = __ldg(p.tileoffset + g);
-            while (am != 0u) {
-                const int cc = __ffs(am) - 1;
-                am &= am - 1u;
-                const unsigned ci_c = __shfl_sync(0xFFFFFFFFu, ci, cc);
-                const float sx_c = __shfl_sync(0xFFFFFFFFu, sx, cc);
-                const unsigned n = ci_c & 0xFFFFu;
-                if (n == 0u) continue;
-                const int64_t slot = g * kTileK + cc;
-                // the 8 bitmap words of the column tile (each lane one, four times over), set bits before each
-                const unsigned wd = __ldg(p.bitmap32 + slot * 8 + (lane & 7));
-                const unsigned cnt = __popc(wd);
-                unsigned inc = cnt;
-                scan8_level<1>(inc);
-                scan8_level<2>(inc);
-                scan8_level<4>(inc);
-                const unsigned w_mine = __shfl_sync(0xFFFFFFFFu, wd, my_word);
-                const unsigned before = __shfl_sync(0xFFFFFFFFu, inc - cnt, my_word);
-                const unsigned bits = (w_mine >> my_shift) & 0xFFu;                 // my 8 rows
-                if (bits != 0u) {
-                    const unsigned rank = before + __popc(w_mine & ((1u << my_shift) - 1u));
-                    const unsigned first = to + (ci_c >> 16);                        // first code of the column tile
-                    if (SPDP_CHECK(p.status, first, (n + 31u) & ~31u, p.codes_len, kSiteValuesSpan) &&
-                        SPDP_CHECK(p.status, rank, 1, n, kSiteRecordIndex)) {
+            const uint32_t* bm = p.bitmap32 + g * (kTileK * 8) + my_word;       // my word of column 0 of the GTile
+            // The active columns are taken 8 at a time in three sweeps, so that the loads of a sweep are
+            // all in flight together: (a) my bitmap word of each column, (b) ranks, then my two code words
+            // of each column, (c) the walks.
+#pragma unroll 1
+            for (int h8 = 0; h8 < kTileK; h8 += 8) {
+                const unsigned sub = (am >> h8) & 0xFFu;                         // warp-uniform
+                if (sub == 0u) continue;
+                unsigned wd[8], w0[8], w1[8], meta[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    if ((sub >> i) & 1u) wd[i] = __ldg(bm + (h8 + i) * 8);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    if (!((sub >> i) & 1u)) continue;
+                    const unsigned ci_c = __shfl_sync(0xFFFFFFFFu, ci, h8 + i);
+                    // set bits before my word: a warp scan in which one lane per word (of the four that hold it) counts
+                    const unsigned cnt = __popc(wd[i]);
+                    unsigned inc = (lane & 3) == 0 ? cnt : 0u;
+#pragma unroll
+                    for (int d = 1; d < 32; d <<= 1) {
+                        const unsigned u = __shfl_up_sync(0xFFFFFFFFu, inc, d);
+                        if (lane >= d) inc += u;
+                    }
+                    const unsigned bits = (wd[i] >> my_shift) & 0xFFu;           // my 8 rows
+                    const unsigned rank = inc - cnt + __popc(wd[i] & ((1u << my_shift) - 1u));
+                    const unsigned first = to + (ci_c >> 16);                     // first code of the column tile
+                    meta[i] = 0u;
+                    if (bits != 0u &&
+                        SPDP_CHECK(p.status, first, ((ci_c & 0xFFFFu) + 31u) & ~31u, p.codes_len, kSiteValuesSpan) &&
+                        SPDP_CHECK(p.status, rank, 1, ci_c & 0xFFFFu, kSiteRecordIndex)) {
                         // my codes: at most 8 nibbles from nibble `rank` on, inside two consecutive 32-bit words
-                        const uint32_t* cw = reinterpret_cast<const uint32_t*>(p.codes + (first >> 1)) + (rank >> 3);
-                        unsigned span = __funnelshift_r(__ldg(cw), __ldg(cw + 1), 4 * (rank & 7u));
+                        const uint32_t* cw = reinterpret_cast<const uint32_t*>(p.codes) + (first >> 3) + (rank >> 3);
+                        w0[i] = __ldg(cw);
+                        w1[i] = __ldg(cw + 1);
+                        meta[i] = bits | ((rank & 7u) << 8);
+                    }
+                }
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    if (!((sub >> i) & 1u)) continue;
+                    const float sx_c = __shfl_sync(0xFFFFFFFFu, sx, h8 + i);
+                    const unsigned bits = meta[i] & 0xFFu;
+                    if (bits != 0u) {
+                        unsigned span = __funnelshift_r(w0[i], w1[i], 4 * (meta[i] >> 8));
+                        // code -> float without a conversion: 0x4B000000 | code is 2^23 + code as a float
 #pragma unroll
                         for (int k = 0; k < 8; ++k) {
-                            if ((bits >> k) & 1u) {
-                                acc[k] = fmaf(static_cast<float>(static_cast<int>(span & 15u) - 8), sx_c, acc[k]);
-                                span >>= 4;
-                            }
+                            const bool on = (bits >> k) & 1u;
+                            const float q = __uint_as_float((span & 15u) | 0x4B000000u) - 8388616.0f;   // code - 8
+                            acc[k] = on ? fmaf(q, sx_c, acc[k]) : acc[k];
+                            span = on ? span >> 4 : span;
                         }
                     }
                 }

@@ -448,3 +448,25 @@ def test_mask_rule_with_the_mask_at_the_end_of_its_allocation(S):
                 check_y(y.cpu().numpy().astype(np.float64), y_ref, S_ref)
             finally:
                 S.spdp_free(h)
+
+
+def test_row_sharded_handles_reproduce_the_product(S):
+    """Row-tile sharding on one GPU: every rank's slice packed as its own matrix, the slices of y side by
+    side against the oracle (the collective that joins them is exercised by the two-rank CPU test)."""
+    w = WL.config4(2304, 1040, seed=12)
+    a = O.active_ref(w.x, w.rule, w.thr)
+    y_ref, S_ref = O.spmspv_ref(w.W, w.x, a)
+    x = dev(w.x)
+    for world in (2, 3, 16):
+        y = torch.full((w.M,), float("nan"), dtype=torch.float32, device="cuda")
+        for rank in range(world):
+            first, rows = S.spdp_row_shard(w.M, world, rank)
+            if rows == 0:
+                continue
+            h = S.spdp_pack_tiled_cbc(dev(w.W[first:first + rows]))
+            try:
+                S.spdp_spmspv(h, x, w.rule, w.thr, y[first:first + rows])
+            finally:
+                torch.cuda.synchronize()
+                S.spdp_free(h)
+        check_y(y.cpu().numpy().astype(np.float64), y_ref, S_ref)

@@ -220,6 +220,21 @@ SPDP_API spdp_status spdp_spmspv_noalloc(const void* tileoffset_dev, const void*
                                 const void* x_dev, spdp_dp_rule rule, float thr, const void* mask_dev,
                                 void* y_dev, spdp_ydtype ydt, void* stream);
 
+/* Producer-fused dynamic pruning (Sec. 6: DP variants that materialise a mask map to the same column
+ * interface; Sec. 4.2 step (3): a magnitude test against a threshold calibrated offline).  The input of
+ * a gated MLP's down-projection is x = silu(gate) * up; this call computes it (fp32 arithmetic, one
+ * rounding to fp16) and writes, in the same pass, the mask of the columns the following spdp_spmspv
+ * should keep: bit (j % 32) of word (j / 32) is NOT(|x_j| <= thr) evaluated on the STORED fp16 x_j, i.e.
+ * exactly the set SPDP_DP_ABS_GT would choose.  Pass the mask with SPDP_DP_MASK.  A caller with
+ * another per-column score (say |x_j| times a column norm) gets its mask from spdp_active_columns on
+ * the score vector and uses SPDP_DP_MASK in the same way.
+ *   gate_dev, up_dev  fp16 [K], device.     x_dev_out  fp16 [K], device.
+ *   mask_dev_out      uint32[ceil(K/32)], device (bits beyond K clear).
+ *   count_dev_out     int32[1], device, or NULL: number of kept columns.
+ * Asynchronous on `stream`; allocates nothing. */
+SPDP_API spdp_status spdp_swiglu_dp(const void* gate_dev, const void* up_dev, int64_t K, float thr, void* x_dev_out,
+                           void* mask_dev_out, void* count_dev_out, void* stream);
+
 /* Row-tile sharding over several GPUs (the paper names multi-GPU execution as future work, Sec. 6; the
  * natural split of y = W x keeps whole 256-row tiles together, so every rank packs its own rows as
  * an independent Tiled-CBC matrix, x is replicated, and the outputs are disjoint).  This is the split

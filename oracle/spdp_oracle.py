@@ -456,6 +456,14 @@ def active_bytes_q4(p: dict, active, y_bytes_per_elem: int = 2) -> int:
     return int(per_tile[:, a].sum()) + 4 * (gt_active + 1) + 2 * K + y_bytes_per_elem * M
 
 
+def swiglu_ref(gate, up) -> np.ndarray:
+    """The activation in front of a gated MLP's down-projection, x = silu(gate) * up with
+    silu(g) = g / (1 + exp(-g)), in fp64 on the exactly widened fp16 inputs.  Returns float64 [K]
+    (a producer kernel rounds it to fp16; the DP decision is then taken on the rounded value)."""
+    g, u = as_f64(gate), as_f64(up)
+    return g / (1.0 + np.exp(-g)) * u
+
+
 def tolerance(S) -> np.ndarray:
     """Per-output bound of the parity gate: 1e-3 * S[i] + 1e-5."""
     return 1e-3 * np.asarray(S, dtype=np.float64) + 1e-5

@@ -420,6 +420,19 @@ spdp_status spdp_spmspv_host(spdp_handle h, const void* x_host, spdp_dp_rule rul
     return SPDP_OK;
 }
 
+spdp_status spdp_swiglu_dp(const void* gate_dev, const void* up_dev, int64_t K, float thr, void* x_dev_out,
+                           void* mask_dev_out, void* count_dev_out, void* stream) {
+    if (gate_dev == nullptr || up_dev == nullptr || x_dev_out == nullptr || mask_dev_out == nullptr) return SPDP_ERR_INVALID_ARG;
+    if (K < 1 || K > (int64_t(1) << 30)) return SPDP_ERR_UNSUPPORTED_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(gate_dev) & 1u) || (reinterpret_cast<uintptr_t>(up_dev) & 1u) ||
+        (reinterpret_cast<uintptr_t>(x_dev_out) & 1u) || (reinterpret_cast<uintptr_t>(mask_dev_out) & 3u) ||
+        (reinterpret_cast<uintptr_t>(count_dev_out) & 3u))
+        return SPDP_ERR_INVALID_ARG;
+    return launch_swiglu_dp(static_cast<const __half*>(gate_dev), static_cast<const __half*>(up_dev), K, thr,
+                            static_cast<__half*>(x_dev_out), static_cast<uint32_t*>(mask_dev_out),
+                            static_cast<int*>(count_dev_out), static_cast<cudaStream_t>(stream));
+}
+
 spdp_status spdp_row_shard(int64_t M, int world, int rank, int64_t* first_row_out, int64_t* rows_out) {
     if (M < 1 || world < 1 || rank < 0 || rank >= world || first_row_out == nullptr || rows_out == nullptr)
         return SPDP_ERR_INVALID_ARG;

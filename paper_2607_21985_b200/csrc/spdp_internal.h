@@ -114,6 +114,10 @@ spdp_status pack_q4_device(spdp_matrix* h, const __half* W, int64_t ldw, cudaStr
 spdp_status launch_spmspv_q4(const spdp_matrix* h, const __half* x, int rule, float thr, const uint32_t* mask, void* y,
                              int ydt, cudaStream_t s);
 
+// producer.cu
+spdp_status launch_swiglu_dp(const __half* gate, const __half* up, int64_t K, float thr, __half* x_out, uint32_t* mask_out,
+                             int* count, cudaStream_t s);
+
 // spmm.cu
 spdp_status configure_spmm_kernel();            // per-device kernel attributes; idempotent
 spdp_status launch_spmm(const spdp_matrix* h, const __half* X, int64_t N, int64_t ldx, void* Y, int64_t ldy, int ydt,

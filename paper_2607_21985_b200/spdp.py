@@ -29,7 +29,7 @@ EXPORTS = (
     "spdp_pack_tiled_cbc", "spdp_pack_tiled_cbc_ex", "spdp_import_tiled_cbc", "spdp_spmspv",
     "spdp_spmspv_host", "spdp_spmspv_noalloc", "spdp_spmspv_batch", "spdp_free", "spdp_get_info", "spdp_export", "spdp_unpack",
     "spdp_active_columns", "spdp_last_device_status", "spdp_set_num_ctas", "spdp_last_cuda_error",
-    "spdp_status_string", "spdp_probe_stream_read", "spdp_probe_gather", "spdp_spmm", "spdp_pack_tiled_cbc_q4", "spdp_export_q4", "spdp_row_shard",
+    "spdp_status_string", "spdp_probe_stream_read", "spdp_probe_gather", "spdp_spmm", "spdp_pack_tiled_cbc_q4", "spdp_export_q4", "spdp_row_shard", "spdp_swiglu_dp",
 )
 
 
@@ -77,6 +77,7 @@ def lib():
         L.spdp_spmm.argtypes = [vp, vp, i64, i64, vp, i64, ci, vp]
         L.spdp_pack_tiled_cbc_q4.argtypes = [vp, i64, i64, i64, ci, ci, vp, ctypes.POINTER(vp)]
         L.spdp_export_q4.argtypes = [vp, vp, vp, vp, vp, vp]
+        L.spdp_swiglu_dp.argtypes = [vp, vp, i64, cf, vp, vp, vp, vp]
         L.spdp_row_shard.argtypes = [i64, ci, ci, ctypes.POINTER(i64), ctypes.POINTER(i64)]
         L.spdp_probe_stream_read.argtypes = [vp, vp]
         L.spdp_probe_gather.argtypes = [vp, vp, ci, cf, vp, vp]
@@ -260,6 +261,14 @@ def spdp_spmm(h: int, X, Y, stream=None) -> None:
     ldy = int(Y.stride(0)) if N > 1 else max(int(Y.shape[1]), int(Y.stride(0)))
     ydt = SPDP_Y_F32 if Y.dtype == torch.float32 else SPDP_Y_F16
     _check(lib().spdp_spmm(h, X.data_ptr(), N, ldx, Y.data_ptr(), ldy, ydt, _stream(stream)), "spdp_spmm")
+
+
+def spdp_swiglu_dp(gate, up, thr: float, x_out, mask_out, count_out=None, stream=None) -> None:
+    """x_out = silu(gate) * up (fp16 CUDA [K]) and the K-bit keep-mask of its columns in one pass."""
+    K = int(gate.shape[0])
+    st = lib().spdp_swiglu_dp(_dev_ptr(gate, "gate"), _dev_ptr(up, "up"), K, float(thr), _dev_ptr(x_out, "x_out"),
+                              _dev_ptr(mask_out, "mask_out"), _dev_ptr(count_out, "count_out", True), _stream(stream))
+    _check(st, "spdp_swiglu_dp")
 
 
 def spdp_row_shard(M: int, world: int, rank: int):

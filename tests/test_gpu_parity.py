@@ -470,3 +470,39 @@ def test_row_sharded_handles_reproduce_the_product(S):
                 torch.cuda.synchronize()
                 S.spdp_free(h)
         check_y(y.cpu().numpy().astype(np.float64), y_ref, S_ref)
+
+
+def test_producer_fused_activation_and_mask(S):
+    """x = silu(gate) * up with the keep-mask written in the same pass: x within one fp16 step of the fp64
+    definition, the mask exactly the set the magnitude rule chooses on the stored x, and the decode call
+    with that mask bit-identical to the decode call that tests x itself."""
+    rng = np.random.Generator(np.random.PCG64(83))
+    M, K = 1536, 3000
+    gate = rng.standard_normal(K).astype(np.float16) * np.float16(2.0)
+    up = rng.standard_normal(K).astype(np.float16)
+    gate[:4] = np.asarray([0.0, -0.0, 30.0, -30.0], np.float16)
+    W = (rng.standard_normal((M, K)) * (rng.random((M, K)) < 0.5) * 0.05).astype(np.float16)
+    thr = 0.3
+    x_out = torch.full((K,), float("nan"), dtype=torch.float16, device="cuda")
+    mask = torch.full(((K + 31) // 32,), -1, dtype=torch.int32, device="cuda")
+    cnt = torch.full((1,), -5, dtype=torch.int32, device="cuda")
+    S.spdp_swiglu_dp(dev(gate), dev(up), thr, x_out, mask, cnt)
+    torch.cuda.synchronize()
+    xg = x_out.cpu().numpy()
+    ref = O.swiglu_ref(gate, up)
+    step = np.maximum(np.abs(ref), 2.0 ** -14) * 2.0 ** -10                  # one fp16 step at that magnitude
+    assert np.all(np.abs(xg.astype(np.float64) - ref) <= step)
+    a = O.active_ref(xg, O.DP_ABS_GT, thr)                                   # decided on the kernel's own fp16 x
+    assert np.array_equal(mask.cpu().numpy().view(np.uint32), O.active_to_words(a)) and int(cnt.item()) == int(a.sum())
+    h = S.spdp_pack_tiled_cbc(dev(W))
+    try:
+        y_mask = torch.empty(M, dtype=torch.float32, device="cuda")
+        y_test = torch.empty(M, dtype=torch.float32, device="cuda")
+        S.spdp_spmspv(h, x_out, O.DP_MASK, 0.0, y_mask, mask=mask)
+        S.spdp_spmspv(h, x_out, O.DP_ABS_GT, thr, y_test)
+        torch.cuda.synchronize()
+        assert np.array_equal(y_mask.cpu().numpy(), y_test.cpu().numpy())
+        y_ref, S_ref = O.spmspv_ref(W, xg, a)
+        check_y(y_mask.cpu().numpy().astype(np.float64), y_ref, S_ref)
+    finally:
+        S.spdp_free(h)

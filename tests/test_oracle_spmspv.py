@@ -245,3 +245,14 @@ def test_spmm_ref_from_packed_arrays_equals_dense():
     Yb, _ = O.spmm_ref(back, X)
     assert np.array_equal(Ya, Yb)
     assert np.allclose(Ya, X.astype(np.float64) @ w.W.astype(np.float64).T, rtol=0, atol=0)   # cross-check only
+
+
+def test_swiglu_ref_on_known_values():
+    g = _f16([0.0, 1.0, -1.0, 20.0, -20.0, 2.0])
+    u = _f16([3.0, 1.0, 1.0, 0.5, 1.0, -2.0])
+    got = O.swiglu_ref(g, u)
+    # silu(1) = 1 / (1 + 1/e) = 0.7310585786300049, silu(-1) = -0.2689414213699951, silu(20) ~ 20, silu(-20) ~ -4.1e-8
+    want = [0.0, 0.7310585786300049, -0.2689414213699951, 20.0 * 0.5 / (1 + np.exp(-20.0)), -20.0 / (1 + np.exp(20.0)),
+            -2.0 * 2.0 / (1 + np.exp(-2.0))]
+    assert np.allclose(got, want, rtol=1e-15, atol=0)
+    assert abs(got[3] - 10.0) < 1e-7 and abs(got[4]) < 5e-8

@@ -83,3 +83,55 @@ def test_full_size_small_batch(S, c_oracle, name, B):
             assert np.all(err <= tol), f"{name} token {b}: worst error/tolerance {np.nanmax(err / tol):.3g}"
     finally:
         S.spdp_free(h)
+
+
+@pytest.mark.parametrize("name,N", [("c1", 16), ("c1", 128), ("c1", 1024), ("c4_rows3584", 128), ("c4_rows3584", 1024)])
+def test_full_size_prefill(S, c_oracle, name, N):
+    """The prefill entry point on benchmark-shaped layers (c1 whole; c4's K = 8192 with 14 of its 112 row
+    tiles, so that the fp64 oracle product stays within seconds): every token of a sample against the C
+    oracle's single-vector result without DP, fp16 outputs as the benchmark uses them."""
+    w = CASES["c1"]() if name == "c1" else WL.config4(M=3584)
+    rng = np.random.Generator(np.random.PCG64(np.random.SeedSequence(600 + N)))
+    X = rng.standard_normal((N, w.K), dtype=np.float32).astype(np.float16)
+    h = S.spdp_pack_tiled_cbc(torch.from_numpy(w.W).cuda())
+    try:
+        Y = torch.full((N, w.M), float("nan"), dtype=torch.float16, device="cuda")
+        S.spdp_spmm(h, torch.from_numpy(X).cuda(), Y)
+        torch.cuda.synchronize()
+        assert S.spdp_last_device_status(h) == 0
+        out = Y.cpu().numpy().astype(np.float64)
+        assert not np.isnan(out).any()
+        every = np.ones(w.K, dtype=bool)
+        for n in sorted(set([0, 1, N // 3, N // 2, N - 2, N - 1]) & set(range(N))):
+            y_ref, S_ref, _ = c_oracle.spmspv(w.W, X[n], every)
+            err = np.abs(out[n] - y_ref)
+            tol = O.tolerance(S_ref)
+            assert np.all(err <= tol), f"{name} token {n}: worst error/tolerance {np.nanmax(err / tol):.3g}"
+    finally:
+        S.spdp_free(h)
+
+
+@pytest.mark.parametrize("name", ["c1", "c3"])
+def test_full_size_q4(S, name):
+    """The 4-bit variant at full size, default CTA count, fp16 y: packed arrays bit for bit against the
+    oracle's, y on the rows of three row tiles against the product on the dequantised weights."""
+    w = CASES[name]()
+    a = O.active_ref(w.x, w.rule, w.thr)
+    want = O.pack_q4_fast(w.W)
+    h = S.spdp_pack_tiled_cbc_q4(torch.from_numpy(w.W).cuda())
+    try:
+        got = S.spdp_export_q4(h)
+        for key in ("tileoffset", "colinfo", "bitmap", "codes", "scales"):
+            assert np.array_equal(got[key], want[key]), key
+        y = torch.full((w.M,), float("nan"), dtype=torch.float16, device="cuda")
+        S.spdp_spmspv(h, torch.from_numpy(w.x).cuda(), w.rule, w.thr, y)
+        torch.cuda.synchronize()
+        assert S.spdp_last_device_status(h) == 0
+        out = y.cpu().numpy().astype(np.float64)
+        R = w.M // 256
+        for r in (0, R // 2, R - 1):
+            sub = O.pack_q4_fast(w.W[256 * r:256 * (r + 1)])
+            y_ref, S_ref = O.spmspv_dense64_ref(O.dequant_q4_ref(sub), w.x, a)
+            assert np.all(np.abs(out[256 * r:256 * (r + 1)] - y_ref) <= O.tolerance(S_ref)), (name, r)
+    finally:
+        S.spdp_free(h)

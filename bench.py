@@ -538,6 +538,92 @@ def run_sharded(args):
         dist.destroy_process_group()
 
 
+def context_legs(args, spdp, torch, w, handles, xs, ys, step, copies, B_active, info, Wd):
+    """Measurements that put the headline in context (none of them is the headline): one call by
+    itself, the same bytes fetched without decoding, a contiguous read of Values, dense fp16 GEMV."""
+    # ---- one call by itself: an unrelated small kernel before every call, so that no call's
+    # prologue overlaps the previous call's tail (the back-to-back figure above is pipelined) ----
+    isolated_us, probes = None, {}
+    if not args.no_context:
+        # Both sequences are replayed from CUDA graphs, so the host's launch rate is out of the picture:
+        # n x (small unrelated kernel, call) against n x (small unrelated kernel).
+        filler = torch.zeros(1 << 16, dtype=torch.float32, device="cuda")
+        n_iso = copies * max(1, -(-60 // copies))
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for i in range(copies):
+                step(i)
+            filler.add_(1.0)
+            side.synchronize()
+            g_both, g_fill = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g_both, stream=side):
+                for i in range(n_iso):
+                    filler.add_(1.0)
+                    step(i)
+            with torch.cuda.graph(g_fill, stream=side):
+                for i in range(n_iso):
+                    filler.add_(1.0)
+            times = {}
+            for name, g in (("both", g_both), ("fill", g_fill)):
+                for _ in range(3):
+                    g.replay()
+                side.synchronize()
+                reps = []
+                for _ in range(5):
+                    a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    a0.record(side)
+                    g.replay()
+                    a1.record(side)
+                    side.synchronize()
+                    reps.append(a0.elapsed_time(a1))
+                times[name] = float(np.median(reps))
+        torch.cuda.current_stream().wait_stream(side)
+        isolated_us = (times["both"] - times["fill"]) / n_iso * 1e3
+        del g_both, g_fill
+
+        # ---- context: the same bytes with plain loads and no decode; a contiguous read of Values ----
+        def timed_probe(fn, n=30):
+            for i in range(2 * copies):
+                fn(i % copies)
+            torch.cuda.synchronize()
+            p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            p0.record()
+            for i in range(n):
+                fn(i % copies)
+            p1.record()
+            torch.cuda.synchronize()
+            return p0.elapsed_time(p1) / n * 1e3
+        g_us = timed_probe(lambda k: spdp.spdp_probe_gather(handles[k], xs[k], w.rule, w.thr))
+        s_us = timed_probe(lambda k: spdp.spdp_probe_stream_read(handles[k]))
+        probes = {"gather_active_tiles_no_decode_us": g_us,
+                  "gather_active_tiles_no_decode_gbs": B_active / g_us / 1e3,
+                  "contiguous_read_of_values_us": s_us,
+                  "contiguous_read_of_values_gbs": 2 * info.values_len / s_us / 1e3}
+
+    # ---- context: dense fp16 GEMV on the same GPU (library kernel, not the product) -------
+    dense_us = None
+    if not args.no_context:
+        try:
+            Wd2 = Wd.clone()
+            Ws = [Wd, Wd2]
+            for i in range(5):
+                torch.mv(Ws[i % 2], xs[0])
+            torch.cuda.synchronize()
+            d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            d0.record()
+            for i in range(50):
+                torch.mv(Ws[i % 2], xs[0])
+            d1.record()
+            torch.cuda.synchronize()
+            dense_us = d0.elapsed_time(d1) / 50 * 1e3
+            del Wd2, Ws
+        except Exception:
+            dense_us = None
+
+    return isolated_us, probes, dense_us
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -621,6 +707,12 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    # ---- context legs first (rank 0): they also bring the GPU to its working state (clocks, TLBs)
+    # before the timed region, which stays exactly `warmup` untimed and `steps` timed calls ----
+    isolated_us, probes, dense_us = None, {}, None
+    if rank == 0:
+        isolated_us, probes, dense_us = context_legs(args, spdp, torch, w, handles, xs, ys, step, copies, B_active, info, Wd)
+    del Wd
     # ---- device-resident timing ---------------------------------------------------------
     sampler.start()
     for i in range(args.warmup):
@@ -693,61 +785,6 @@ def main():
             dist.barrier()
             dist.destroy_process_group()
         return
-
-    # ---- one call by itself: an unrelated small kernel before every call, so that no call's
-    # prologue overlaps the previous call's tail (the back-to-back figure above is pipelined) ----
-    isolated_us = None
-    probes = {}
-    if not args.no_context:
-        filler = torch.zeros(1 << 16, dtype=torch.float32, device="cuda")
-        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(60)]
-        for i, (a0, a1) in enumerate(evs):
-            filler.add_(1.0)
-            a0.record()
-            step(i)
-            a1.record()
-        torch.cuda.synchronize()
-        isolated_us = float(np.median([a0.elapsed_time(a1) for a0, a1 in evs[10:]])) * 1e3
-
-        # ---- context: the same bytes with plain loads and no decode; a contiguous read of Values ----
-        def timed_probe(fn, n=30):
-            for i in range(2 * copies):
-                fn(i % copies)
-            torch.cuda.synchronize()
-            p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            p0.record()
-            for i in range(n):
-                fn(i % copies)
-            p1.record()
-            torch.cuda.synchronize()
-            return p0.elapsed_time(p1) / n * 1e3
-        g_us = timed_probe(lambda k: spdp.spdp_probe_gather(handles[k], xs[k], w.rule, w.thr))
-        s_us = timed_probe(lambda k: spdp.spdp_probe_stream_read(handles[k]))
-        probes = {"gather_active_tiles_no_decode_us": g_us,
-                  "gather_active_tiles_no_decode_gbs": B_active / g_us / 1e3,
-                  "contiguous_read_of_values_us": s_us,
-                  "contiguous_read_of_values_gbs": 2 * info.values_len / s_us / 1e3}
-
-    # ---- context: dense fp16 GEMV on the same GPU (library kernel, not the product) -------
-    dense_us = None
-    if not args.no_context:
-        try:
-            Wd2 = Wd.clone()
-            Ws = [Wd, Wd2]
-            for i in range(5):
-                torch.mv(Ws[i % 2], xs[0])
-            torch.cuda.synchronize()
-            d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            d0.record()
-            for i in range(50):
-                torch.mv(Ws[i % 2], xs[0])
-            d1.record()
-            torch.cuda.synchronize()
-            dense_us = d0.elapsed_time(d1) / 50 * 1e3
-            del Wd2, Ws
-        except Exception:
-            dense_us = None
-    del Wd
 
     peak, peak_kind = measured_peak()
     launch_us = ms_per_step * 1e3

@@ -4,15 +4,17 @@
 // (its "layout alignment" stage: TILE_K_PAD stride, ldmatrix.x4, mma.m16n8k16), and accumulates
 // there.  On Blackwell the tensor cores read both operands straight from shared memory
 // (tcgen05.mma) and accumulate in tensor memory, so the layout-alignment stage becomes the decode
-// itself: every thread writes the dense fp16 values of its row, 8 columns at a time, directly at
-// the address the operand descriptor expects (K-major core matrices of 8 rows x 16 bytes, no
-// swizzle).  No registers hold accumulators and no ldmatrix pass exists.
+// itself: W is given to the tensor cores M-major (rows contiguous), which is how a column tile
+// lies in Tiled-CBC, so a lane that owns 8 consecutive rows of a column (one bitmap byte: its
+// values are one contiguous run, rank = set bits before the byte, Sec. 4.2.1) writes exactly one
+// 16-byte piece of the operand tile per column.  No registers hold accumulators, no ldmatrix pass.
 //
-// One CTA = one row tile (256 rows = two M = 128 accumulators) x kNT tokens, walking all of K in
-// blocks of 64 columns (4 GTiles): copy the 64 column tiles (compressed) and the X tile into shared
-// memory, decode, issue 2 x 4 tcgen05.mma (K = 16 each), commit them to a shared-memory barrier.
-// Two CTAs share an SM (each owns half of tensor memory), so one decodes while the other's
-// tensor-core work runs.  The only wait (on that barrier) is bounded.
+// One CTA = one row tile (256 rows = two M = 128 accumulators) x kNT tokens (all 512 columns of
+// tensor memory), walking K in blocks of kKB columns through a software pipeline: while the
+// tensor cores multiply block k, the warps decode block k+1, and the copies of the compressed
+// column tiles of block k+2 and of the X tile of block k+1 are in flight.  A warp copies and decodes
+// its own columns, so the compressed data needs no CTA-wide barrier; one barrier per block precedes
+// the tensor-core issue.  The only waits (on the tensor cores' completion barriers) are bounded.
 #include <cstddef>
 #include <mutex>
 
@@ -24,15 +26,28 @@ namespace {
 
 using namespace dev;
 
-constexpr int kThreads = 256;          // 8 warps; warp w decodes rows 32w .. 32w+31 of the row tile (bitmap word w)
-constexpr int kKB = 64;                // columns per K-block: 4 GTiles, 4 tensor-core steps of K = 16
-constexpr int kNT = 128;               // tokens per CTA (the N of the tensor-core instruction)
-constexpr int kTmemCols = 2 * kNT;     // two accumulators of 128 rows x kNT fp32 columns (a power of two >= 32)
-constexpr int kCoreBytes = 128;        // a core matrix: 8 rows x 16 bytes, rows 16 bytes apart
-constexpr int kRowGroupBytes = (kKB / 8) * kCoreBytes;   // the 8 core matrices of 8 rows, one after the other along K
-constexpr int kHalfBytes = 16 * kRowGroupBytes;          // 128 rows
+constexpr int kWarps = 16;             // warp w decodes columns w, w + 16 of a K-block; lane l owns rows 8l .. 8l+7
+constexpr int kThreads = kWarps * 32;
+constexpr int kKB = 64;                // columns per K-block: 4 GTiles, 4 tensor-core steps of K = 16 per accumulator
+constexpr int kNT = 256;               // tokens per CTA (the N of the tensor-core instruction)
+constexpr int kTmemCols = 2 * kNT;     // two accumulators of 128 rows x kNT fp32 columns
+constexpr int kAStages = 2, kBStages = 2, kCStages = 2;
+// A (decoded W), M-major without swizzle: 16-byte piece = 8 consecutive rows of one column; the 8
+// columns of a k-group are 16 bytes apart (a core matrix of 128 bytes), the 16 row chunks of a
+// 128-row half 144 bytes apart (128 + 16: the 16-byte pieces that the lanes of a quarter warp store for
+// one column then fall into different banks), the k-groups 16 * 144 bytes apart.
+constexpr int kAChunkStride = 144;                 // stride byte offset: next 8 rows
+constexpr int kAKGroupStride = 16 * kAChunkStride; // leading byte offset: next 8 columns
+constexpr int kAHalfBytes = (kKB / 8) * kAKGroupStride;
+// B (X tile), K-major without swizzle: 16-byte piece = 8 consecutive columns of one token; the 8 tokens
+// of a group are 16 bytes apart, the k-groups 128 bytes apart, the token groups kKB/8 * 128 bytes apart.
+constexpr int kBCore = 128;
+constexpr int kBTokenGroupStride = (kKB / 8) * kBCore;
+constexpr int kBBytes = (kNT / 8) * kBTokenGroupStride;
 constexpr int kWaitTries = 1 << 22;
-static_assert(kTmemCols == 256 || kTmemCols == 512 || kTmemCols == 128, "tensor memory is allocated in powers of two");
+static_assert(kTmemCols == 512, "the CTA owns all of tensor memory");
+static_assert(kKB % 16 == 0 && kKB % kWarps == 0, "whole columns per warp and K-block");
+constexpr int kColsPerWarp = kKB / kWarps;
 
 struct Params {
     const uint32_t* tileoffset;
@@ -51,32 +66,32 @@ struct Params {
     int64_t values_len;
 };
 
+struct CompStage {                              // one K-block as stored: compact values, bitmaps
+    alignas(16) unsigned short vals[kKB][kTileM];
+    alignas(16) uint32_t bm[kKB][8];
+};
 struct __align__(128) Smem {
-    unsigned char A[2][kHalfBytes];                 // decoded W: [half][row group][k core][row in group][8 fp16]
-    unsigned char B[(kNT / 8) * kRowGroupBytes];    // X tile:    [token group][k core][token in group][8 fp16]
-    alignas(16) unsigned short vals[kKB][kTileM];   // the K-block's column tiles as stored (compact values)
-    alignas(16) uint32_t bm[kKB][8];                // their bitmaps as 32-bit words
-    unsigned short prefix[kKB][8];                  // set bits before each word inside its column tile
-    uint32_t start[kKB];                            // start of each column tile's values in Values (elements)
-    uint32_t pieces[kKB];                           // its 16-byte pieces
-    alignas(8) unsigned long long mma_done;         // the tensor cores' completion barrier
+    unsigned char A[kAStages][2][kAHalfBytes];  // decoded W, two 128-row halves per stage
+    unsigned char B[kBStages][kBBytes];         // X tiles
+    CompStage comp[kCStages];
+    alignas(8) unsigned long long mma_done[kAStages];   // the tensor cores are done with A stage s (and the B stage used with it)
     uint32_t tmem_base;
     int abort;
 };
-static_assert(sizeof(Smem) <= 110 * 1024, "two CTAs per SM");
+static_assert(sizeof(Smem) <= 227 * 1024, "shared memory of one CTA");
 
-// Shared-memory operand descriptor of tcgen05.mma for a K-major tile without swizzle: the 16-byte
-// row pieces of 8 consecutive rows are contiguous (a core matrix); lbo = distance between the two
-// core matrices one instruction reads along K, sbo = distance between 8-row groups.
+// Shared-memory operand descriptor of tcgen05.mma, no swizzle: start address, leading byte offset,
+// stride byte offset (all in 16-byte units), descriptor version of this architecture.
 __device__ __forceinline__ uint64_t operand_desc(uint32_t smem_addr, uint32_t lbo, uint32_t sbo) {
     uint64_t d = (smem_addr & 0x3FFFFu) >> 4;
     d |= static_cast<uint64_t>(lbo >> 4) << 16;
     d |= static_cast<uint64_t>(sbo >> 4) << 32;
-    d |= static_cast<uint64_t>(1) << 46;            // descriptor version of this architecture
-    return d;                                       // layout type 0 (no swizzle), base offset 0
+    d |= static_cast<uint64_t>(1) << 46;
+    return d;
 }
-// Instruction descriptor: fp16 x fp16 -> fp32, both operands K-major, M = 128, N = kNT.
-constexpr uint32_t kInstrDesc = (1u << 4) | (static_cast<uint32_t>(kNT >> 3) << 17) | (static_cast<uint32_t>(128 >> 4) << 24);
+// Instruction descriptor: fp16 x fp16 -> fp32, A M-major (bit 15), B K-major, M = 128, N = kNT.
+constexpr uint32_t kInstrDesc = (1u << 4) | (1u << 15) | (static_cast<uint32_t>(kNT >> 3) << 17) |
+                                (static_cast<uint32_t>(128 >> 4) << 24);
 
 __device__ __forceinline__ void mma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, bool accumulate) {
     asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
@@ -94,7 +109,36 @@ __device__ __forceinline__ bool wait_parity(unsigned long long* bar, unsigned pa
     return false;
 }
 
-__global__ void __launch_bounds__(kThreads, 2)
+// The 8 rows of one column tile that lane `lane` owns (one bitmap byte), as 8 fp16 in row order, zeros
+// where the bit is clear.  The set bits before each of the 8 bitmap words come from a scan over
+// 8-lane segments (every segment holds the 8 words); rank = those + the bits below the lane's byte;
+// then a walk over the byte (Sec. 4.2.1).
+__device__ __forceinline__ uint4 decode_chunk(const CompStage& cs, int j, int lane) {
+    const unsigned w8 = cs.bm[j][lane & 7];
+    const unsigned cnt = __popc(w8);
+    unsigned inc = cnt;
+    scan8_level<1>(inc);
+    scan8_level<2>(inc);
+    scan8_level<4>(inc);
+    const unsigned word = __shfl_sync(0xFFFFFFFFu, w8, lane >> 2);
+    const unsigned before = __shfl_sync(0xFFFFFFFFu, inc - cnt, lane >> 2);
+    const int sh = 8 * (lane & 3);
+    const unsigned bits = (word >> sh) & 0xFFu;
+    unsigned out[4] = {0u, 0u, 0u, 0u};
+    if (bits != 0u) {
+        const unsigned short* v = &cs.vals[j][before + __popc(word & ((1u << sh) - 1u))];
+#pragma unroll
+        for (int r = 0; r < 8; ++r) {
+            if ((bits >> r) & 1u) {
+                out[r >> 1] |= static_cast<unsigned>(*v) << (16 * (r & 1));
+                ++v;
+            }
+        }
+    }
+    return make_uint4(out[0], out[1], out[2], out[3]);
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
 spmm_kernel(const __grid_constant__ Params p) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     Smem& sm = *reinterpret_cast<Smem*>(smem_raw);
@@ -103,9 +147,11 @@ spmm_kernel(const __grid_constant__ Params p) {
     const int nb = static_cast<int>(blockIdx.x - static_cast<unsigned>(r) * static_cast<unsigned>(p.nblocks));
     const int64_t n0 = static_cast<int64_t>(nb) * kNT;
 
-    // ---- set-up: the completion barrier, and this CTA's half of tensor memory ----
+    // ---- set-up: the completion barriers, and tensor memory ----
     if (t == 0) {
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&sm.mma_done)) : "memory");
+#pragma unroll
+        for (int s = 0; s < kAStages; ++s)
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&sm.mma_done[s])) : "memory");
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         sm.abort = 0;
     }
@@ -118,110 +164,126 @@ spmm_kernel(const __grid_constant__ Params p) {
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem = sm.tmem_base;
+    const int nkb = (p.C * kTileK + kKB - 1) / kKB;
 
-    const uint32_t a_base = smem_u32(&sm.A[0][0]), b_base = smem_u32(&sm.B[0]);
-    const uint32_t vals_base = smem_u32(&sm.vals[0][0]), bm_base = smem_u32(&sm.bm[0][0]);
-    const int nkb = (p.C + 3) / 4;
-    const unsigned lt_mask = (1u << lane) - 1u;
-    bool ok = true;
-
-    for (int kb = 0; kb < nkb; ++kb) {
-        // ---- (1) where the K-block's 64 column tiles are (ColInfo, TileOffset: Sec. 4.1) ----
-        if (t < kKB) {
-            const int gc = 4 * kb + (t >> 4);                                   // GTile column
-            uint32_t start = 0, pieces = 0;
-            if (gc < p.C) {
-                const int64_t g = static_cast<int64_t>(r) * p.C + gc;
-                const uint32_t ci = __ldg(p.colinfo + g * kTileK + (t & 15));
-                start = __ldg(p.tileoffset + g) + (ci >> 16);
-                pieces = ((ci & 0xFFFFu) + 7u) >> 3;
-                if (!SPDP_CHECK(p.status, start, 8u * pieces, p.values_len, kSiteValuesSpan) ||
+    // Where the column tiles this warp handles in K-block kb lie (ColInfo, TileOffset: Sec. 4.1): lane q < 4
+    // looks up column warp + 16 q.  The loads are issued one iteration before their values are needed.
+    struct Meta { uint32_t ci, to; };
+    auto fetch_meta = [&](int kb) -> Meta {
+        Meta m = {0u, 0u};
+        const int col = kb * kKB + warp + kWarps * lane;
+        if (lane < kColsPerWarp && kb < nkb && (col >> 4) < p.C) {
+            const int64_t g = static_cast<int64_t>(r) * p.C + (col >> 4);
+            m.ci = __ldg(p.colinfo + g * kTileK + (col & 15));
+            m.to = __ldg(p.tileoffset + g);
+        }
+        return m;
+    };
+    // Starts the copies of this warp's column tiles of K-block kb as stored: lane l the l-th 16-byte piece
+    // of the values, lanes 0-1 the bitmap.
+    auto load_comp = [&](int kb, const Meta m) {
+        if (kb >= nkb) return;
+        CompStage& cs = sm.comp[kb % kCStages];
+#pragma unroll
+        for (int q = 0; q < kColsPerWarp; ++q) {
+            const int j = warp + kWarps * q;
+            const int col = kb * kKB + j;
+            const uint32_t ci = __shfl_sync(0xFFFFFFFFu, m.ci, q), to = __shfl_sync(0xFFFFFFFFu, m.to, q);
+            if ((col >> 4) < p.C) {
+                const int64_t slot = (static_cast<int64_t>(r) * p.C + (col >> 4)) * kTileK + (col & 15);
+                const uint32_t start = to + (ci >> 16);
+                int pieces = static_cast<int>(((ci & 0xFFFFu) + 7u) >> 3);
+                if (!SPDP_CHECK(p.status, start, 8 * pieces, p.values_len, kSiteValuesSpan) ||
                     !SPDP_CHECK(p.status, 0, pieces, 32, kSitePieces))
-                    pieces = 0;                                                 // checked build only: the tile is left out
-            }
-            sm.start[t] = start;
-            sm.pieces[t] = pieces;
-        }
-        __syncthreads();
-        // ---- (2) copy them, and the X tile, into shared memory (16-byte asynchronous copies) ----
-        {
-            const int j = t >> 2, sub = t & 3;
-            const int gc = 4 * kb + (j >> 4);
-            const int pieces = static_cast<int>(sm.pieces[j]);
-            const unsigned char* src = reinterpret_cast<const unsigned char*>(p.values) + 2ull * sm.start[j];
-            for (int pc = sub; pc < pieces; pc += 4) cp_async16<0>(vals_base + j * (2 * kTileM) + 16 * pc, src + 16 * pc, 1);
-            if (sub < 2) {
-                if (gc < p.C) {
-                    const int64_t slot = (static_cast<int64_t>(r) * p.C + gc) * kTileK + (j & 15);
-                    cp_async16<0>(bm_base + 32 * j + 16 * sub, reinterpret_cast<const unsigned char*>(p.bitmap) + 32 * slot + 16 * sub, 1);
-                } else {
-                    *reinterpret_cast<uint4*>(&sm.bm[j][4 * sub]) = make_uint4(0u, 0u, 0u, 0u);   // beyond the last GTile column
+                    pieces = -1;                                                 // checked build only: the tile is left out
+                if (lane < pieces)
+                    cp_async16<0>(smem_u32(&cs.vals[j][8 * lane]), reinterpret_cast<const unsigned char*>(p.values) + 2ull * start + 16 * lane, 1);
+                if (lane < 2) {
+                    if (pieces >= 0)
+                        cp_async16<0>(smem_u32(&cs.bm[j][4 * lane]), reinterpret_cast<const unsigned char*>(p.bitmap) + 32 * slot + 16 * lane, 1);
+                    else
+                        *reinterpret_cast<uint4*>(&cs.bm[j][4 * lane]) = make_uint4(0u, 0u, 0u, 0u);
                 }
+            } else if (lane < 2) {
+                *reinterpret_cast<uint4*>(&cs.bm[j][4 * lane]) = make_uint4(0u, 0u, 0u, 0u);   // beyond the last GTile column
             }
-#pragma unroll
-            for (int i = 0; i < kNT * 8 / kThreads; ++i) {
-                const int c = t + i * kThreads, nl = c >> 3, kc = c & 7;
-                const int64_t n = n0 + nl;
-                const int64_t k = static_cast<int64_t>(kb) * kKB + 8 * kc;
-                int bytes = 0;                                                  // tokens beyond N and columns beyond K read as 0
-                if (n < p.N && k < p.K) bytes = static_cast<int>(min(static_cast<int64_t>(16), 2 * (p.K - k)));
-                const __half* xs = bytes ? p.X + n * p.ldx + k : p.X;
-                cp_async16_partial(b_base + (nl >> 3) * kRowGroupBytes + kc * kCoreBytes + (nl & 7) * 16, xs, bytes);
-            }
-            cp_async_commit();
         }
-        cp_async_wait<0>();
-        __syncthreads();
-        // ---- (3) set bits before each 32-bit word of each column tile ----
+    };
+    // Starts the copies of the X tile of K-block kb: kNT tokens x kKB/8 pieces of 16 bytes, zero beyond N and K.
+    auto load_x = [&](int kb) {
+        if (kb >= nkb) return;
+        const uint32_t b_base = smem_u32(&sm.B[kb % kBStages][0]);
 #pragma unroll
-        for (int e = t; e < kKB * 8; e += kThreads) {
-            const int j = e >> 3, w = e & 7;
-            unsigned pre = 0;
-            for (int q = 0; q < w; ++q) pre += __popc(sm.bm[j][q]);
-            sm.prefix[j][w] = static_cast<unsigned short>(pre);
+        for (int i = 0; i < kNT * (kKB / 8) / kThreads; ++i) {
+            const int c = t + i * kThreads, nl = c % kNT, kc = c / kNT;         // consecutive threads: consecutive tokens
+            const int64_t n = n0 + nl;
+            const int64_t k = static_cast<int64_t>(kb) * kKB + 8 * kc;
+            int bytes = 0;
+            if (n < p.N && k < p.K) bytes = static_cast<int>(min(static_cast<int64_t>(16), 2 * (p.K - k)));
+            const __half* xs = bytes ? p.X + n * p.ldx + k : p.X;
+            cp_async16_partial(b_base + (nl >> 3) * kBTokenGroupStride + kc * kBCore + (nl & 7) * 16, xs, bytes);
         }
-        __syncthreads();
-        // ---- (4) decode (Sec. 4.2.1 / 4.3): my row's value in each of the 64 columns, rank = set bits
-        // before my position; 8 columns make one 16-byte piece of the operand tile ----
+    };
+
+    // A wait that runs out (it never should) clears `ok`: the thread then stops waiting but keeps
+    // walking the same barriers as the others, the status word gets SPDP_ERR_TIMEOUT and the outputs stay unwritten.
+    bool ok = true;
+    // copy groups: G(-2) = {comp(0), X(0)}, G(-1) = {comp(1)}, then G(kb) = {comp(kb+2), X(kb+1)} at the end of block kb
+    load_comp(0, fetch_meta(0));
+    load_x(0);
+    cp_async_commit();
+    load_comp(1, fetch_meta(1));
+    cp_async_commit();
+    Meta meta_next = fetch_meta(2);
+    for (int kb = 0; kb < nkb; ++kb) {
+        const int sa = kb % kAStages;
+        cp_async_wait<1>();                 // my column tiles of block kb have arrived (the newest group may be in flight)
+        __syncwarp();
+        const CompStage& cs = sm.comp[kb % kCStages];
+        // the tensor cores must be done with this A stage (block kb - kAStages)
+        if (kb >= kAStages && ok) ok = wait_parity(&sm.mma_done[sa], ((kb / kAStages) - 1) & 1);
+        // ---- decode: my 8 rows of my columns, one 16-byte piece each ----
         {
-            const uint32_t a_row = a_base + (warp >> 2) * kHalfBytes + ((warp & 3) * 4 + (lane >> 3)) * kRowGroupBytes + (lane & 7) * 16;
-#pragma unroll 2
-            for (int kc = 0; kc < 8; ++kc) {
-                unsigned out[4] = {0u, 0u, 0u, 0u};
+            unsigned char* a_stage = &sm.A[sa][lane >> 4][0] + (lane & 15) * kAChunkStride;
 #pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    const int j = 8 * kc + c;
-                    const unsigned word = sm.bm[j][warp];
-                    unsigned v = 0;
-                    if ((word >> lane) & 1u) v = sm.vals[j][sm.prefix[j][warp] + __popc(word & lt_mask)];
-                    out[c >> 1] |= v << (16 * (c & 1));
-                }
-                asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};"
-                             ::"r"(a_row + kc * kCoreBytes), "r"(out[0]), "r"(out[1]), "r"(out[2]), "r"(out[3]) : "memory");
+            for (int q = 0; q < kColsPerWarp; ++q) {
+                const int j = warp + q * kWarps;
+                const uint4 piece = decode_chunk(cs, j, lane);
+                *reinterpret_cast<uint4*>(a_stage + (j >> 3) * kAKGroupStride + (j & 7) * 16) = piece;
             }
         }
+        cp_async_wait<0>();                 // my pieces of the X tile of block kb have arrived
         // the operand tiles were written through the generic proxy; the tensor cores read through the async proxy
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncthreads();
-        // ---- (5) one thread issues the K-block's tensor-core work and commits it to the barrier ----
+        // ---- one thread issues the K-block's tensor-core work and commits it to the stage's barrier ----
         if (t == 0) {
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t a_base = smem_u32(&sm.A[sa][0][0]), b_base = smem_u32(&sm.B[kb % kBStages][0]);
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
 #pragma unroll
                 for (int kk = 0; kk < kKB / 16; ++kk) {
-                    const uint64_t ad = operand_desc(a_base + h * kHalfBytes + kk * 2 * kCoreBytes, kCoreBytes, kRowGroupBytes);
-                    const uint64_t bd = operand_desc(b_base + kk * 2 * kCoreBytes, kCoreBytes, kRowGroupBytes);
+                    const uint64_t ad = operand_desc(a_base + h * kAHalfBytes + kk * 2 * kAKGroupStride, kAKGroupStride, kAChunkStride);
+                    const uint64_t bd = operand_desc(b_base + kk * 2 * kBCore, kBCore, kBTokenGroupStride);
                     mma_f16(tmem + h * kNT, ad, bd, kb > 0 || kk > 0);
                 }
             }
             asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
-                         ::"r"(smem_u32(&sm.mma_done)) : "memory");
+                         ::"r"(smem_u32(&sm.mma_done[sa])) : "memory");
         }
-        // ---- (6) the tiles may be overwritten once the tensor cores are done with them ----
-        ok = wait_parity(&sm.mma_done, kb & 1);
-        if (!ok) break;
+        // Next copies: my column tiles of block kb+2 go where I just decoded block kb from; the X tile of
+        // block kb+1 goes into the stage block kb-1 multiplied from, once that work is known to be complete.
+        load_comp(kb + 2, meta_next);
+        meta_next = fetch_meta(kb + 3);
+        if (kb >= 1 && kb + 1 < nkb && ok) ok = wait_parity(&sm.mma_done[(kb - 1) % kAStages], ((kb - 1) / kAStages) & 1);
+        load_x(kb + 1);
+        cp_async_commit();
     }
+    // the last blocks' tensor-core work
+    for (int kb = (nkb > kAStages ? nkb - kAStages : 0); ok && kb < nkb; ++kb)
+        ok = wait_parity(&sm.mma_done[kb % kAStages], (kb / kAStages) & 1);
+    cp_async_wait<0>();
     if (!ok) {
         sm.abort = 1;
         if (lane == 0) atomicCAS(p.status, 0, SPDP_ERR_TIMEOUT);
@@ -229,12 +291,14 @@ spmm_kernel(const __grid_constant__ Params p) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     __syncthreads();
 
-    // ---- epilogue: tensor memory -> registers -> Y.  Warp w reads lanes 32*(w%4).. of accumulator w/4;
-    // a thread holds one row, 16 tokens at a time, so a warp's stores of one token are 32 consecutive rows ----
+    // ---- epilogue: tensor memory -> registers -> Y.  Warp w reads lanes 32*(w%4).. of accumulator (w/4)%2,
+    // token columns [(w/8)*kNT/2, +kNT/2); a thread holds one row, 16 tokens at a time, so a warp's stores of
+    // one token are 32 consecutive rows ----
     if (!sm.abort) {
-        const int half = warp >> 2, lane_base = 32 * (warp & 3);
+        const int half = (warp >> 2) & 1, lane_base = 32 * (warp & 3), cbase = (warp >> 3) * (kNT / 2);
         const int64_t row = static_cast<int64_t>(r) * kTileM + half * 128 + lane_base + lane;
-        for (int c0 = 0; c0 < kNT; c0 += 16) {
+        for (int c0 = cbase; c0 < cbase + kNT / 2; c0 += 16) {
+            if (n0 + c0 >= p.N) break;                                          // warp-uniform
             uint32_t v[16];
             asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
                          : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),

@@ -40,8 +40,10 @@ constexpr int kAChunkStride = 144;                 // stride byte offset: next 8
 constexpr int kAKGroupStride = 16 * kAChunkStride; // leading byte offset: next 8 columns
 constexpr int kAHalfBytes = (kKB / 8) * kAKGroupStride;
 // B (X tile), K-major without swizzle: 16-byte piece = 8 consecutive columns of one token; the 8 tokens
-// of a group are 16 bytes apart, the k-groups 128 bytes apart, the token groups kKB/8 * 128 bytes apart.
-constexpr int kBCore = 128;
+// of a group are 16 bytes apart (a core matrix of 128 bytes), the k-groups 144 bytes apart (128 + 16: a warp
+// copies 4 tokens x 8 k-groups per instruction, 4 whole lines of X, and its 32 pieces then spread evenly
+// over the banks), the token groups kKB/8 * 144 bytes apart.
+constexpr int kBCore = 144;
 constexpr int kBTokenGroupStride = (kKB / 8) * kBCore;
 constexpr int kBBytes = (kNT / 8) * kBTokenGroupStride;
 constexpr int kWaitTries = 1 << 22;
@@ -215,7 +217,7 @@ spmm_kernel(const __grid_constant__ Params p) {
         const uint32_t b_base = smem_u32(&sm.B[kb % kBStages][0]);
 #pragma unroll
         for (int i = 0; i < kNT * (kKB / 8) / kThreads; ++i) {
-            const int c = t + i * kThreads, nl = c % kNT, kc = c / kNT;         // consecutive threads: consecutive tokens
+            const int c = t + i * kThreads, nl = c / (kKB / 8), kc = c % (kKB / 8);   // 8 consecutive threads: one token's 128 bytes
             const int64_t n = n0 + nl;
             const int64_t k = static_cast<int64_t>(kb) * kKB + 8 * kc;
             int bytes = 0;

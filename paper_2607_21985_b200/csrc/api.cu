@@ -99,6 +99,8 @@ spdp_status finish_handle(spdp_matrix* h) {
     if (st != SPDP_OK) return st;
     st = configure_spmm_kernel();
     if (st != SPDP_OK) return st;
+    st = configure_spmspv_q4_kernel();
+    if (st != SPDP_OK) return st;
     SPDP_CUDA_TRY(cudaMalloc(&h->status_word, 2 * sizeof(int)));
     SPDP_CUDA_TRY(cudaMemset(h->status_word, 0, 2 * sizeof(int)));
     SPDP_CUDA_TRY(cudaMalloc(&h->x_stage, h->K * sizeof(__half)));

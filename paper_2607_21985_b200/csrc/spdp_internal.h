@@ -110,6 +110,7 @@ spdp_status launch_spmspv_batch(const spdp_matrix* h, const __half* x, int64_t l
                                 cudaStream_t s);
 
 // spmspv_q4.cu / pack.cu: the 4-bit variant
+spdp_status configure_spmspv_q4_kernel();      // per-device kernel attributes; idempotent
 spdp_status pack_q4_device(spdp_matrix* h, const __half* W, int64_t ldw, cudaStream_t s);
 spdp_status launch_spmspv_q4(const spdp_matrix* h, const __half* x, int rule, float thr, const uint32_t* mask, void* y,
                              int ydt, cudaStream_t s);

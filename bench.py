@@ -161,7 +161,7 @@ class ClockSampler:
         use = self.timed_samples if len(self.timed_samples) >= 3 else self.samples
         return {"sm_mhz": float(np.median(use)) if use else None, "sm_max_mhz": self.max_mhz,
                 "reasons": sorted(self.reasons), "samples": len(use),
-                "window": "timed" if use is self.timed_samples else "warmup+timed"}
+                "window": "timed" if use is self.timed_samples else "context legs + warm-up + timed (the timed region is too short for 3 samples)"}
 
 
 def cpu_baseline(w, B_active_full, gpu=None):
@@ -709,12 +709,12 @@ def main():
 
     # ---- context legs first (rank 0): they also bring the GPU to its working state (clocks, TLBs)
     # before the timed region, which stays exactly `warmup` untimed and `steps` timed calls ----
+    sampler.start()                      # clocks are sampled from here on: context legs, warm-up, timed region
     isolated_us, probes, dense_us = None, {}, None
     if rank == 0:
         isolated_us, probes, dense_us = context_legs(args, spdp, torch, w, handles, xs, ys, step, copies, B_active, info, Wd)
     del Wd
     # ---- device-resident timing ---------------------------------------------------------
-    sampler.start()
     for i in range(args.warmup):
         step(i)
     barrier()

@@ -380,7 +380,7 @@ def run_prefill(args):
         "warmup": args.warmup, "ms_per_step": us * 1e-3, "us_per_call": us, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f16 in, f32 accumulate", "data": "synthetic",
         "config": {"workload": w.name, "tokens": N, "nnz": int(info.nnz), "packed_bytes": int(info.packed_bytes),
-                   "l2": "X, Y and the packed matrix exceed L2 together; W is re-read once per block of 128 tokens"},
+                   "l2": "X, Y and the packed matrix exceed L2 together; W is decoded once per block of 256 or 512 tokens"},
         "gpu_launches": steps,
         "roofline": {"bound": "tensor", "achieved": issued, "peak": peak, "unit": "TFLOP/s", "frac": issued / peak,
                      "peak_kind": f"of {peak_kind}", "traffic": None, "kernel": "spmm_kernel",

@@ -44,7 +44,7 @@ typedef enum {
     SPDP_ERR_ALLOC = -3,             /* device or host allocation failed                        */
     SPDP_ERR_CUDA = -4,              /* a CUDA runtime call failed (see spdp_last_cuda_error)    */
     SPDP_ERR_OVERFLOW = -5,          /* Values would need 2^32 or more elements (TileOffset is 32-bit) */
-    SPDP_ERR_TIMEOUT = -6            /* reserved: a bounded device-side wait expired (no kernel waits today) */
+    SPDP_ERR_TIMEOUT = -6            /* a bounded device-side wait expired (spdp_spmm; see spdp_last_device_status) */
 } spdp_status;
 
 /* Dynamic-pruning rule: which columns of W are fetched for this x (Sec. 2.2 "Dynamic Pruning",
@@ -174,14 +174,16 @@ SPDP_API spdp_status spdp_spmspv_batch(spdp_handle h, const void* x_dev, int64_t
  * the paper's layout-alignment stage does for its tensor-core path), the contraction runs on the
  * 5th-generation tensor cores (tcgen05.mma, fp16 inputs, fp32 accumulation in tensor memory).
  *   X_dev   fp16 [N][ldx], device, one token per row, ldx >= K elements between tokens; X_dev must
- *           be 16-byte aligned and ldx a multiple of 8 (the tiles are copied in 16-byte pieces),
- *           else SPDP_ERR_INVALID_ARG.
+ *           be 16-byte aligned and ldx a multiple of 8 (the tiles are read through a tensor map,
+ *           encoded on the host at every call), else SPDP_ERR_INVALID_ARG.
  *   N       >= 1 tokens.
  *   Y_dev   [N][ldy] of ydt, device, ldy >= M elements between tokens; all N*M entries are written.
  * Asynchronous on `stream`, allocates nothing, launches one kernel; no split along K, so no
- * workspace is touched and calls on one handle may overlap.  The waits inside the kernel (on the
- * tensor cores' completion barrier) are bounded; one that runs out records SPDP_ERR_TIMEOUT in the
- * handle's status word and the CTA leaves its outputs unwritten. */
+ * workspace is touched and calls on one handle may overlap.  The waits inside the kernel (on
+ * shared-memory barriers that the copies and the tensor cores complete) are bounded; one that runs
+ * out records SPDP_ERR_TIMEOUT in the handle's status word and the CTA leaves its outputs unwritten;
+ * TileOffset words that do not describe a K-block that fits shared memory record SPDP_ERR_OVERFLOW
+ * the same way.  SPDP_ERR_CUDA if the driver's tensor-map encoder cannot be found. */
 SPDP_API spdp_status spdp_spmm(spdp_handle h, const void* X_dev, int64_t N, int64_t ldx, void* Y_dev, int64_t ldy,
                       spdp_ydtype ydt, void* stream);
 

@@ -49,7 +49,8 @@ WORKER = textwrap.dedent("""
     assert y.shape[0] == w.M and np.array_equal(y.numpy(), y_ref), "gathered result differs from the unsharded one"
     y2 = sh.spmspv(torch.from_numpy(w.x))                           # buffers are reused from call to call
     assert np.array_equal(y2.numpy(), y_ref)
-    print("rank", dist.get_rank(), "rows", sh.rows, "ok")
+    sys.stdout.write("rank %d rows %d SHARD_OK\n" % (dist.get_rank(), sh.rows))          # one write per rank: lines do not interleave
+    sys.stdout.flush()
     dist.destroy_process_group()
 """)
 
@@ -66,4 +67,4 @@ def test_two_gloo_ranks_gather_the_unsharded_result(tmp_path, M):
            "--master-port", str(port), str(script)]
     out = subprocess.run(cmd, capture_output=True, text=True, timeout=600)
     assert out.returncode == 0, out.stdout[-2000:] + out.stderr[-2000:]
-    assert out.stdout.count(" ok") == 2
+    assert out.stdout.count("SHARD_OK") == 2

@@ -49,7 +49,7 @@ WORKER = textwrap.dedent("""
     assert y.shape[0] == w.M and np.array_equal(y.numpy(), y_ref), "gathered result differs from the unsharded one"
     y2 = sh.spmspv(torch.from_numpy(w.x))                           # buffers are reused from call to call
     assert np.array_equal(y2.numpy(), y_ref)
-    sys.stdout.write("rank %d rows %d SHARD_OK\n" % (dist.get_rank(), sh.rows))          # one write per rank: lines do not interleave
+    sys.stdout.write("rank %d rows %d SHARD_OK\\n" % (dist.get_rank(), sh.rows))          # one write per rank: lines do not interleave
     sys.stdout.flush()
     dist.destroy_process_group()
 """)

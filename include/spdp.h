@@ -74,7 +74,7 @@ typedef struct {
     const void* colinfo_dev;     /* uint32[NGT*16] (column start inside its GTile) << 16 | nnz   */
     const void* bitmap_dev;      /* uint64[NGT*16*4] bit b of word w = row 64*w+b of the column tile */
     const void* values_dev;      /* fp16[values_len] nonzeros in tile-column order, zero padded  */
-    int32_t num_ctas;          /* CTAs one spdp_spmspv launches (see spdp_set_num_ctas)         */
+    int32_t num_ctas;          /* CTAs one spdp_spmspv launches                                 */
     int32_t device;            /* CUDA device ordinal the handle lives on                       */
 } spdp_info;
 
@@ -286,19 +286,9 @@ SPDP_API spdp_status spdp_probe_gather(spdp_handle h, const void* x_dev, spdp_dp
  * Synchronises the device. */
 SPDP_API spdp_status spdp_last_device_status(spdp_handle h, int* out);
 
-/* Tuning knob: how spdp_spmspv splits the matrix over CTAs.  Takes effect on the next call; re-derives the
- * handle's split-K workspace (may reallocate it, always empties it).
- *   n > 0   the GTiles in storage order are cut into n equal contiguous ranges, one CTA each (at most 1024 and
- *           at most one per GTile are used); row tiles that several CTAs feed are combined through the workspace
- *           (Sec. 4.2 step 6 across CTAs).
- *   n = 0   the default: one such CTA per SM.
- *   n = -S  (S = 2..8) "row-tile clusters": one thread-block cluster of S CTAs per row tile, each CTA taking 1/S of
- *           the row tile's GTiles, the S partial sums added in rank order through the cluster's shared memory (no
- *           workspace traffic).  fp16 Values and the single-vector call only (the other kernels keep the default
- *           ranges).  Falls back to smaller S, then to the default ranges, if R clusters of that size are not
- *           resident at once.  For small matrices whose R * S CTAs still cover most SMs.
- * Results are bit-identical from call to call for a given setting; different settings add in different orders.
- * SPDP_ERR_INVALID_ARG for n < -8 or n = -1. */
+/* Tuning knob: number of CTAs spdp_spmspv launches (0 = default, one per SM; at most 1024 and at
+ * most one per GTile are used).  Takes effect on
+ * the next call; re-derives the handle's split-K workspace layout (may reallocate it). */
 SPDP_API spdp_status spdp_set_num_ctas(spdp_handle h, int num_ctas);
 
 /* Text of the last CUDA runtime error seen by the library on this thread ("" if none). */

@@ -78,22 +78,6 @@ spdp_status build_partition(spdp_matrix* h, int num_ctas) {
     cudaFree(h->workspace);     h->workspace = nullptr;
     cudaFree(h->workspace_batch);   h->workspace_batch = nullptr;
     h->num_ctas = P;
-    // Row-tile clusters (asked for with a negative count): the fp16 single-vector kernel then runs one cluster of S
-    // CTAs per row tile and adds the CTAs' shares through the cluster's shared memory instead of the split-K tree.
-    // Only if all R clusters are resident at once; otherwise a smaller S, then the ranges.  Never the default: on
-    // the small layers it measured 0.4-0.7 us faster per call in graph replay and no faster back to back.
-    h->cluster_s = 0;
-    if (!h->q4 && h->pad_elems == 8 && num_ctas < 0) {
-        int S = -num_ctas;
-        if (S > spmspv_max_cluster_size()) S = spmspv_max_cluster_size();
-        if (S > h->C) S = static_cast<int>(h->C);
-        for (; S >= 2; --S) {
-            if (spmspv_max_active_clusters(S) >= h->R) {
-                h->cluster_s = S;
-                break;
-            }
-        }
-    }
     h->workspace_bytes = static_cast<int64_t>(P) * kTileM * sizeof(float);   // one row of split-K tree nodes per CTA
     SPDP_CUDA_TRY(cudaMalloc(&h->workspace, h->workspace_bytes));
     SPDP_CUDA_TRY(cudaMemset(h->workspace, 0, h->workspace_bytes));
@@ -488,7 +472,7 @@ spdp_status spdp_get_info(spdp_handle h, spdp_info* out) {
     i.colinfo_dev = h->colinfo;
     i.bitmap_dev = h->bitmap;
     i.values_dev = h->values;
-    i.num_ctas = h->cluster_s > 1 ? static_cast<int32_t>(h->R) * h->cluster_s : h->num_ctas;
+    i.num_ctas = h->num_ctas;
     i.device = h->device;
     *out = i;
     return SPDP_OK;
@@ -552,7 +536,7 @@ spdp_status spdp_last_device_status(spdp_handle h, int* out) {
 }
 
 spdp_status spdp_set_num_ctas(spdp_handle h, int num_ctas) {
-    if (!valid(h) || num_ctas < -8 || num_ctas == -1) return SPDP_ERR_INVALID_ARG;
+    if (!valid(h) || num_ctas < 0) return SPDP_ERR_INVALID_ARG;
     SPDP_CUDA_TRY(cudaDeviceSynchronize());
     return build_partition(h, num_ctas);
 }

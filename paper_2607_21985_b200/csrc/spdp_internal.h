@@ -37,7 +37,6 @@ struct spdp_matrix {
     // Work partition of one spmspv launch: the kernel cuts the NGT GTiles into num_ctas equal
     // contiguous ranges, one per CTA.
     int num_ctas;           // P
-    int cluster_s;          // > 1: spdp_spmspv (fp16 Values) launches R clusters of cluster_s CTAs, one per row tile, instead
     float* workspace;       // device [P*256] split-K tree nodes, one row per CTA (all zero between calls)
     float* workspace_batch; // device [P*8*256] tree nodes of the small-batch call (all zero between calls)
     int* status_word;       // device [2]: the status word, and a sink word the benchmark probes may write
@@ -98,8 +97,6 @@ spdp_status unpack_device(const spdp_matrix* h, __half* W, int64_t ldw, cudaStre
 // spmspv.cu
 int default_ctas_per_sm();   // CTAs of the spMspV kernel that share one SM
 spdp_status configure_spmspv_kernel();   // per-device kernel attributes; idempotent
-int spmspv_max_active_clusters(int cluster_s);   // clusters of that many CTAs of the spMspV kernel resident at once
-int spmspv_max_cluster_size();
 spdp_status launch_spmspv(const spdp_matrix* h, const __half* x, int rule, float thr,
                           const uint32_t* mask, void* y, int ydt, cudaStream_t s);
 spdp_status launch_spmspv_noalloc(const uint32_t* tileoffset, const uint32_t* colinfo, const uint64_t* bitmap,

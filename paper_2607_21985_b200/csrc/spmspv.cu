@@ -64,7 +64,6 @@ struct Params {
     int M, K, R, C;
     int64_t NGT;            // R * C GTiles, cut into num_ctas equal contiguous ranges
     int num_ctas;
-    int cluster_s;          // > 1: the launch is R clusters of cluster_s CTAs, one cluster per row tile (no workspace)
     float* workspace;       // [num_ctas][256] tree nodes of the split-K combine, all zero between calls
     int* status;
     int64_t values_len;     // elements of Values (the checked build holds every fetch against it)
@@ -105,8 +104,6 @@ static_assert(sizeof(uint32_t) * (kChunkCols + kChunkGT) + 2 * kChunkCols + size
 static_assert(sizeof(Smem) <= (227 * 1024) / kCtasPerSm - 1024 * (kCtasPerSm - 1), "shared memory of one CTA");
 static_assert(kRecPad <= kThreads, "one thread per trailing null record");
 static_assert(kWarps >= 16, "two groups of 256 threads finish two row tiles side by side");
-constexpr int kMaxClusterS = 8;             // row-tile clusters: CTAs per cluster (the portable limit)
-static_assert(kMaxClusterS <= kWarps, "a cluster's shares fit the buffer that parks a first row tile");
 
 // DP test of Sec. 4.2 step (3): magnitude against the threshold; NOT(|x| <= thr) keeps NaN.
 __device__ __forceinline__ bool column_active(int rule, float thr, const uint32_t* mask, int j, __half xj) {
@@ -186,17 +183,6 @@ __device__ __forceinline__ void finish_row_tile(const Params& p, int r, const fl
         store_y(p.y, p.ydt, row, part);
 }
 
-// Row-tile clusters: adds the kWarps per-warp partial sums of my share of the row tile in warp order and leaves
-// the result in slot `crank` of the buffer at `slots` in the shared memory of the cluster's first CTA.
-__device__ __forceinline__ void deposit_row_tile(const float (*red)[kTileM], float* slots, unsigned crank, int tt) {
-    float part = 0.f;
-#pragma unroll
-    for (int w = 0; w < kWarps; ++w) part += red[w][tt];
-    uint32_t remote;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(smem_u32(slots + crank * kTileM + tt)), "r"(0));
-    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(part) : "memory");
-}
-
 // One persistent CTA per GTile range; every warp runs its own fetch -> decode pipeline.
 // The range is cut into pieces (part of one row tile, at most kChunkGT GTiles).  A batch is one
 // piece, or the last piece of a row tile together with the first piece of the next row tile, so
@@ -220,19 +206,7 @@ spmspv_kernel(const Params p) {
     Smem& sm = *reinterpret_cast<Smem*>(smem_raw);
 
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
-    // My GTile range: one of num_ctas equal pieces of the whole matrix, or (row-tile clusters) piece `crank` of the
-    // cluster_s equal pieces of row tile blockIdx.x / cluster_s.
-    const bool clustered = p.cluster_s > 1;
-    const unsigned crank = clustered ? blockIdx.x % static_cast<unsigned>(p.cluster_s) : 0u;
-    unsigned g_begin, g_end;
-    if (clustered) {
-        const unsigned base = (blockIdx.x / static_cast<unsigned>(p.cluster_s)) * static_cast<unsigned>(p.C);
-        g_begin = base + (static_cast<unsigned>(p.C) * crank) / static_cast<unsigned>(p.cluster_s);
-        g_end = base + (static_cast<unsigned>(p.C) * (crank + 1u)) / static_cast<unsigned>(p.cluster_s);
-    } else {
-        g_begin = range_begin(p, blockIdx.x);
-        g_end = range_begin(p, blockIdx.x + 1);
-    }
+    const unsigned g_begin = range_begin(p, blockIdx.x), g_end = range_begin(p, blockIdx.x + 1);
 
     const int lane7 = lane & 7;
     const int lgrp = lane >> 3;
@@ -546,30 +520,9 @@ spmspv_kernel(const Params p) {
         // batch; the other warps go straight on to the next batch's list phase.  Neither red[] nor
         // red_first[] is written again before these threads have passed the next __syncthreads.
         if (t < kTileM) {
-            if (done_last) {
-                if (clustered) deposit_row_tile(sm.red, &sm.red_first[0][0], crank, t);
-                else finish_row_tile(p, two ? rB : rA, sm.red, t);
-            }
+            if (done_last) finish_row_tile(p, two ? rB : rA, sm.red, t);
         } else if (t < 2 * kTileM) {
             if (two) finish_row_tile(p, rA, sm.red_first, t - kTileM);
-        }
-    }
-    if (clustered) {
-        // ---- row-tile clusters: every CTA has left its share of the row tile in the first CTA's shared memory;
-        // after the cluster's barrier the first CTA adds the shares in rank order and stores the rows ----
-        asm volatile("barrier.cluster.arrive.release.aligned;\n barrier.cluster.wait.acquire.aligned;" ::: "memory");
-        if (crank == 0u && t < kTileM) {
-            if (!waited_for_stream) asm volatile("griddepcontrol.wait;" ::: "memory");      // y may belong to the previous kernel
-            const int r = static_cast<int>(blockIdx.x / static_cast<unsigned>(p.cluster_s));
-            const int64_t row = static_cast<int64_t>(r) * kTileM + t;
-            float sum = 0.f;
-            for (unsigned q = 0; q < static_cast<unsigned>(p.cluster_s); ++q) {
-                const unsigned b = (static_cast<unsigned>(p.C) * q) / static_cast<unsigned>(p.cluster_s);
-                const unsigned e = (static_cast<unsigned>(p.C) * (q + 1u)) / static_cast<unsigned>(p.cluster_s);
-                if (b < e) sum += sm.red_first[0][q * kTileM + t];        // CTAs with an empty range left nothing
-            }
-            if (SPDP_CHECK(p.status, row, 1, static_cast<int64_t>(p.R) * kTileM, kSiteOutputRow) && row < p.M)
-                store_y(p.y, p.ydt, row, sum);
         }
     }
 }
@@ -587,18 +540,11 @@ spdp_status launch_kernel(const Params& p, int num_ctas, cudaStream_t s) {
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = sizeof(Smem);
     cfg.stream = s;
-    cudaLaunchAttribute attr[2];
+    cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (p.cluster_s > 1) {                              // row-tile clusters: one cluster of cluster_s CTAs per row tile
-        attr[1].id = cudaLaunchAttributeClusterDimension;
-        attr[1].val.clusterDim.x = static_cast<unsigned>(p.cluster_s);
-        attr[1].val.clusterDim.y = 1;
-        attr[1].val.clusterDim.z = 1;
-        cfg.numAttrs = 2;
-    }
     SPDP_CUDA_TRY(cudaLaunchKernelEx(&cfg, spmspv_kernel, p));
     return SPDP_OK;
 }
@@ -657,29 +603,6 @@ spdp_status configure_spmspv_kernel() {
     return SPDP_OK;
 }
 
-// How many clusters of `cluster_s` CTAs of the kernel the current device runs at once (0 on any error).
-int spmspv_max_active_clusters(int cluster_s) {
-    if (configure_spmspv_kernel() != SPDP_OK) return 0;
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(static_cast<unsigned>(cluster_s));
-    cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = sizeof(Smem);
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = static_cast<unsigned>(cluster_s);
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, spmspv_kernel, &cfg) != cudaSuccess) {
-        (void)cudaGetLastError();
-        return 0;
-    }
-    return n;
-}
-int spmspv_max_cluster_size() { return kMaxClusterS; }
-
 spdp_status launch_spmspv(const spdp_matrix* h, const __half* x, int rule, float thr,
                           const uint32_t* mask, void* y, int ydt, cudaStream_t s) {
     Params p;
@@ -699,11 +622,10 @@ spdp_status launch_spmspv(const spdp_matrix* h, const __half* x, int rule, float
     p.C = static_cast<int>(h->C);
     p.NGT = h->NGT;
     p.num_ctas = h->num_ctas;
-    p.cluster_s = h->cluster_s;
     p.workspace = h->workspace;
     p.status = h->status_word;
     p.values_len = h->values_len;
-    return launch_kernel(p, h->cluster_s > 1 ? static_cast<int>(h->R) * h->cluster_s : h->num_ctas, s);
+    return launch_kernel(p, h->num_ctas, s);
 }
 
 spdp_status launch_spmspv_noalloc(const uint32_t* tileoffset, const uint32_t* colinfo, const uint64_t* bitmap,
@@ -754,7 +676,6 @@ spdp_status launch_spmspv_noalloc(const uint32_t* tileoffset, const uint32_t* co
     p.C = static_cast<int>(C);
     p.NGT = NGT;
     p.num_ctas = P;
-    p.cluster_s = 0;
     p.workspace = sc->workspace;            // addresses inside the device array (no host dereference)
     p.status = &sc->status;
     p.values_len = int64_t(1) << 40;        // the caller owns Values; its length is not known here

@@ -46,7 +46,7 @@ def test_checked_build_parity_and_clean_status(S, M, K, sp, skip, seed):
     Y_ref, S_ref = O.spmspv_batch_ref(W, X, acts)
     h = S.spdp_pack_tiled_cbc(dev(W))
     try:
-        for ctas in (0, 3, 37, -3, -8):            # default, two range splits, row-tile clusters
+        for ctas in (0, 3, 37):
             S.spdp_set_num_ctas(h, ctas)
             y = torch.full((M,), float("nan"), dtype=torch.float32, device="cuda")
             S.spdp_spmspv(h, dev(X[0]), rule, thr, y)

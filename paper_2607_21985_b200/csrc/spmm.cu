@@ -124,6 +124,12 @@ __device__ __forceinline__ void arrive(unsigned long long* bar) {
 }
 __device__ __forceinline__ bool wait_parity(unsigned long long* bar, unsigned parity) {
     const uint32_t a = smem_u32(bar);
+    {   // the phase is usually complete already: a test costs less than a wait that may suspend
+        unsigned done;
+        asm volatile("{\n .reg .pred p;\n mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+                     : "=r"(done) : "r"(a), "r"(parity) : "memory");
+        if (done) return true;
+    }
     for (int tries = 0; tries < kWaitTries; ++tries) {
         unsigned done;
         asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"

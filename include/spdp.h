@@ -178,8 +178,11 @@ SPDP_API spdp_status spdp_spmspv_batch(spdp_handle h, const void* x_dev, int64_t
  *           encoded on the host at every call), else SPDP_ERR_INVALID_ARG.
  *   N       >= 1 tokens.
  *   Y_dev   [N][ldy] of ydt, device, ldy >= M elements between tokens; all N*M entries are written.
- * Asynchronous on `stream`, allocates nothing, launches one kernel; no split along K, so no
- * workspace is touched and calls on one handle may overlap.  The waits inside the kernel (on
+ * Asynchronous on `stream`.  Usually one kernel and no allocation.  When the last round of CTAs would
+ * leave more than half of the SMs idle, the tiles of that round are cut along K instead: a second launch
+ * leaves fp32 partial sums in scratch memory taken from the device's stream-ordered pool (cudaMallocAsync /
+ * cudaFreeAsync on `stream`, 0.5 MB per slice) and a third adds the slices in a fixed order.  The handle's
+ * workspace is never touched, so calls on one handle may overlap.  The waits inside the kernel (on
  * shared-memory barriers that the copies and the tensor cores complete) are bounded; one that runs
  * out records SPDP_ERR_TIMEOUT in the handle's status word and the CTA leaves its outputs unwritten;
  * TileOffset words that do not describe a K-block that fits shared memory record SPDP_ERR_OVERFLOW

@@ -31,6 +31,7 @@
 // The launch picks the one with fewer rounds of CTAs x cost per K-block (small N: the first).
 #include <cuda.h>
 
+#include <algorithm>
 #include <cstddef>
 #include <mutex>
 
@@ -78,6 +79,10 @@ struct Params {
     int ydt;
     int M, K, C;
     int nblocks;            // token blocks: CTA (or CTA pair) = row tile * nblocks + token block
+    // CTA-pair kernel only: pair i works on tile tile0 + i / kslices, on slice i % kslices of the tile's K-blocks; with
+    // kslices > 1 it leaves fp32 partial sums in partial[i][token in tile][row in tile] instead of writing Y.
+    int tile0, kslices;
+    float* partial;
     int* status;
     int64_t values_len;
 };
@@ -260,6 +265,23 @@ __device__ __forceinline__ void store_accumulators(const Params& p, uint32_t tme
                 if (n < p.N) store_y(p.Y, p.ydt, n * p.ldy + row, __uint_as_float(v[i]));
             }
         }
+    }
+}
+
+// The same for a slice of K: the accumulators go, as fp32, to dst[column * 256 + row] (row = my row inside the row tile).
+__device__ __forceinline__ void store_partial(float* dst, uint32_t tmem, int lane_base, int c_begin, int c_end, int row,
+                                              int valid_columns) {
+    for (int c0 = c_begin; c0 < c_end; c0 += 16) {
+        if (c0 >= valid_columns) break;                                     // warp-uniform
+        uint32_t v[16];
+        asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+                     : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                       "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+                     : "r"(tmem + (static_cast<uint32_t>(lane_base) << 16) + c0) : "memory");
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+            if (c0 + i < valid_columns) dst[static_cast<size_t>(c0 + i) * kTileM + row] = __uint_as_float(v[i]);
     }
 }
 
@@ -498,8 +520,10 @@ spmm_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
     const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
     const int c = static_cast<int>(blockIdx.x & 1u);                  // my rank in the pair = my half of the row tile
     const unsigned pr = blockIdx.x >> 1;
-    const int r = static_cast<int>(pr / static_cast<unsigned>(p.nblocks));
-    const int nb = static_cast<int>(pr - static_cast<unsigned>(r) * static_cast<unsigned>(p.nblocks));
+    const unsigned tile = static_cast<unsigned>(p.tile0) + pr / static_cast<unsigned>(p.kslices);
+    const int slice = static_cast<int>(pr % static_cast<unsigned>(p.kslices));
+    const int r = static_cast<int>(tile / static_cast<unsigned>(p.nblocks));
+    const int nb = static_cast<int>(tile - static_cast<unsigned>(r) * static_cast<unsigned>(p.nblocks));
     const int64_t n0 = static_cast<int64_t>(nb) * kNT;
     const int ntiles = (p.N - n0 > kNI) ? 2 : 1;                      // accumulators in use
 
@@ -527,7 +551,10 @@ spmm_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
     pair_sync();                       // both CTAs' barriers and tensor memory exist before either reaches into the other
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem = sm.tmem_base;
-    const int nkb = (p.C + kGTB - 1) / kGTB;
+    // my K-blocks: slice `slice` of the tile's nkb_all; kb below counts from the slice's first block kb0
+    const int nkb_all = (p.C + kGTB - 1) / kGTB;
+    const int kb0 = static_cast<int>(static_cast<int64_t>(nkb_all) * slice / p.kslices);
+    const int nkb = static_cast<int>(static_cast<int64_t>(nkb_all) * (slice + 1) / p.kslices) - kb0;
     // A wait that runs out (it never should) clears `ok`: the thread then stops waiting but keeps walking the
     // same barriers as the others, the status word gets SPDP_ERR_TIMEOUT and the outputs stay unwritten.
     bool ok = true;
@@ -567,18 +594,18 @@ spmm_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
                 unsigned long long* bar = &sm.ready[kb % kStages];
                 expect_bytes(bar, static_cast<uint32_t>(ntiles) * kBTileBytes);
                 for (int i = 0; i < ntiles; ++i)
-                    tensor_copy(&sm.B[kb % kStages][i * kBTileBytes], &xmap, kb * kKB, static_cast<int>(n0) + i * kNI + c * (kNI / 2), bar);
+                    tensor_copy(&sm.B[kb % kStages][i * kBTileBytes], &xmap, (kb0 + kb) * kKB, static_cast<int>(n0) + i * kNI + c * (kNI / 2), bar);
             };
             for (int kb = 0; kb < kCStages && kb < nkb; ++kb)
-                ok = load_comp(p, r, kb, fetch_offsets(p, r, nkb, kb), sm.comp[kb % kCStages], &sm.comp_full[kb % kCStages]) && ok;
+                ok = load_comp(p, r, kb0 + kb, fetch_offsets(p, r, nkb_all, kb0 + kb), sm.comp[kb % kCStages], &sm.comp_full[kb % kCStages]) && ok;
             for (int kb = 0; kb < kStages && kb < nkb; ++kb) load_x(kb);
-            Offsets next = fetch_offsets(p, r, nkb, kCStages);
+            Offsets next = fetch_offsets(p, r, nkb_all, kb0 + kCStages);
             for (int kb = 0; kb < nkb; ++kb) {
                 // the stored block kb + kCStages goes where block kb was decoded from, once my decode warps are done with it
                 if (kb + kCStages < nkb) {
                     if (ok) ok = wait_parity(&sm.a_ready[kb % kStages], (kb / kStages) & 1);
-                    ok = load_comp(p, r, kb + kCStages, next, sm.comp[kb % kCStages], &sm.comp_full[kb % kCStages]) && ok;
-                    next = fetch_offsets(p, r, nkb, kb + kCStages + 1);
+                    ok = load_comp(p, r, kb0 + kb + kCStages, next, sm.comp[kb % kCStages], &sm.comp_full[kb % kCStages]) && ok;
+                    next = fetch_offsets(p, r, nkb_all, kb0 + kb + kCStages + 1);
                 }
                 // my X tiles of block kb + 1 go where block kb + 1 - kStages multiplied from, once that work is complete
                 const int kx = kb + 1;
@@ -607,7 +634,7 @@ spmm_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
             const unsigned phase = (kb / kStages) & 1;
             if (ok) ok = wait_parity(&sm.comp_full[kb % kCStages], (kb / kCStages) & 1);    // the stored block has arrived
             if (kb >= kStages && ok) ok = wait_parity(&sm.mma_done[s], phase ^ 1u);         // the tensor cores are done with this A stage
-            decode_block(p, sm.comp[kb % kCStages], min(kGTB, p.C - kGTB * kb), c, warp, lane, &sm.A[s][0]);
+            decode_block(p, sm.comp[kb % kCStages], min(kGTB, p.C - kGTB * (kb0 + kb)), c, warp, lane, &sm.A[s][0]);
             // the operand tile was written through the generic proxy; the tensor cores read through the async proxy
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
@@ -630,14 +657,38 @@ spmm_kernel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMa
     // ---- epilogue.  Warp w reads lanes 32*(w%4).. (my rows 32*(w%4)..), token columns [(w/4)*128, +128) of the 512 ----
     if (!sm.abort && warp < kWarps) {
         const int lane_base = 32 * (warp & 3), cbase = (warp >> 2) * (kNT / 4);
-        store_accumulators(p, tmem, lane_base, cbase, cbase + kNT / 4,
-                           static_cast<int64_t>(r) * kTileM + c * 128 + lane_base + lane, n0);
+        if (p.partial == nullptr)
+            store_accumulators(p, tmem, lane_base, cbase, cbase + kNT / 4,
+                               static_cast<int64_t>(r) * kTileM + c * 128 + lane_base + lane, n0);
+        else
+            store_partial(p.partial + static_cast<size_t>(pr) * kNT * kTileM, tmem, lane_base, cbase, cbase + kNT / 4,
+                          c * 128 + lane_base + lane, static_cast<int>(min(static_cast<int64_t>(kNT), p.N - n0)));
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     pair_sync();                       // neither CTA leaves, or frees tensor memory, while the other may still reach into it
     if (warp == 0)
         asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "n"(kTmemCols) : "memory");
+}
+
+// Adds the K-slices of the tiles that were cut along K, in slice order, and writes their part of Y.
+__global__ void reduce_slices_kernel(const Params p, int tiles) {
+    const int64_t total = static_cast<int64_t>(tiles) * kNT * kTileM;
+    for (int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < total;
+         i += static_cast<int64_t>(gridDim.x) * blockDim.x) {
+        const int row_in = static_cast<int>(i % kTileM);
+        const int col = static_cast<int>((i / kTileM) % kNT);
+        const int tt = static_cast<int>(i / (static_cast<int64_t>(kTileM) * kNT));
+        const unsigned tile = static_cast<unsigned>(p.tile0 + tt);
+        const int r = static_cast<int>(tile / static_cast<unsigned>(p.nblocks));
+        const int nb = static_cast<int>(tile - static_cast<unsigned>(r) * static_cast<unsigned>(p.nblocks));
+        const int64_t n = static_cast<int64_t>(nb) * kNT + col, row = static_cast<int64_t>(r) * kTileM + row_in;
+        if (n >= p.N || row >= p.M) continue;
+        const float* src = p.partial + (static_cast<size_t>(tt) * p.kslices * kNT + col) * kTileM + row_in;
+        float sum = 0.f;
+        for (int sl = 0; sl < p.kslices; ++sl) sum += src[static_cast<size_t>(sl) * kNT * kTileM];
+        store_y(p.Y, p.ydt, n * p.ldy + row, sum);
+    }
 }
 
 }  // namespace pair
@@ -709,37 +760,71 @@ spdp_status launch_spmm(const spdp_matrix* h, const __half* X, int64_t N, int64_
     p.C = static_cast<int>(h->C);
     p.status = h->status_word;
     p.values_len = h->values_len;
-    // Which kernel: rounds of CTAs over the SMs x the measured cost of a K-block (a pair's CTA decodes half as much: 3 : 4).
+    p.tile0 = 0;
+    p.kslices = 1;
+    p.partial = nullptr;
+    // Which kernel: rounds of CTAs over the SMs x the measured cost of a K-block (a pair's CTA decodes half as much:
+    // 3 : 4).  A last round of the pair kernel that would hold at most half the pairs is cut along K instead: its
+    // tiles are spread over all pairs as K-slices that leave fp32 partial sums in scratch memory, and a small
+    // kernel adds the slices in order (so the result does not depend on timing).
     const int64_t sms = h->sm_count > 0 ? h->sm_count : 1;
+    const int64_t slots = sms / 2 > 0 ? sms / 2 : 1;                         // pairs resident at once
     const int64_t ctas_one = h->R * ((N + one::kNT - 1) / one::kNT);
-    const int64_t ctas_pair = 2 * h->R * ((N + pair::kNT - 1) / pair::kNT);
-    const bool use_pair = 3 * ((ctas_pair + sms - 1) / sms) < 4 * ((ctas_one + sms - 1) / sms);
-    const int64_t ctas = use_pair ? ctas_pair : ctas_one;
-    if (ctas >= (int64_t(1) << 31)) return SPDP_ERR_UNSUPPORTED_SHAPE;
+    const int64_t tiles = h->R * ((N + pair::kNT - 1) / pair::kNT);         // pair tiles
+    const int64_t nkb = (h->C + kGTB - 1) / kGTB;
+    const int64_t full = (tiles / slots) * slots, rest = tiles - full;
+    int64_t slices = 1;
+    if (full > 0 && rest > 0 && 2 * rest <= slots) slices = std::min<int64_t>(std::min<int64_t>(slots / rest, nkb), 64);
+    const double cost_pair = 3.0 * (static_cast<double>(full / slots) + (rest > 0 ? 1.0 / static_cast<double>(slices) : 0.0) +
+                                    (slices > 1 ? 0.1 : 0.0));
+    const double cost_one = 4.0 * static_cast<double>((ctas_one + sms - 1) / sms);
+    const bool use_pair = cost_pair < cost_one;
+    if (std::max(ctas_one, 2 * tiles * slices) >= (int64_t(1) << 31)) return SPDP_ERR_UNSUPPORTED_SHAPE;
     CUtensorMap xmap;
     spdp_status st = encode_x(&xmap, X, N, h->K, ldx, use_pair ? kNI / 2 : one::kNT);
     if (st != SPDP_OK) return st;
     if (!use_pair) {
         p.nblocks = static_cast<int>((N + one::kNT - 1) / one::kNT);
-        one::spmm_kernel<<<static_cast<unsigned>(ctas), one::kThreads, one::kSmemBytes, s>>>(p, xmap);
+        one::spmm_kernel<<<static_cast<unsigned>(ctas_one), one::kThreads, one::kSmemBytes, s>>>(p, xmap);
         SPDP_CUDA_TRY(cudaGetLastError());
         return SPDP_OK;
     }
     p.nblocks = static_cast<int>((N + pair::kNT - 1) / pair::kNT);
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(static_cast<unsigned>(ctas));
-    cfg.blockDim = dim3(pair::kThreads);
-    cfg.dynamicSmemBytes = pair::kSmemBytes;
-    cfg.stream = s;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 2;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    SPDP_CUDA_TRY(cudaLaunchKernelEx(&cfg, pair::spmm_kernel, p, xmap));
-    return SPDP_OK;
+    auto launch_pairs = [&](int64_t pairs) -> spdp_status {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(static_cast<unsigned>(2 * pairs));
+        cfg.blockDim = dim3(pair::kThreads);
+        cfg.dynamicSmemBytes = pair::kSmemBytes;
+        cfg.stream = s;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        SPDP_CUDA_TRY(cudaLaunchKernelEx(&cfg, pair::spmm_kernel, p, xmap));
+        return SPDP_OK;
+    };
+    if (slices == 1) return launch_pairs(tiles);
+    // whole tiles first, then the last tiles cut along K, then the sum of their slices
+    st = launch_pairs(full);
+    if (st != SPDP_OK) return st;
+    float* scratch = nullptr;
+    const size_t scratch_bytes = static_cast<size_t>(rest * slices) * pair::kNT * kTileM * sizeof(float);
+    SPDP_CUDA_TRY(cudaMallocAsync(reinterpret_cast<void**>(&scratch), scratch_bytes, s));     // stream-ordered, from the device's pool
+    p.tile0 = static_cast<int>(full);
+    p.kslices = static_cast<int>(slices);
+    p.partial = scratch;
+    st = launch_pairs(rest * slices);
+    if (st == SPDP_OK) {
+        const int64_t elems = rest * pair::kNT * kTileM;
+        pair::reduce_slices_kernel<<<static_cast<unsigned>(std::min<int64_t>((elems + 255) / 256, 4096)), 256, 0, s>>>(
+            p, static_cast<int>(rest));
+        if (cudaGetLastError() != cudaSuccess) st = SPDP_ERR_CUDA;
+    }
+    cudaFreeAsync(scratch, s);
+    return st;
 }
 
 }  // namespace spdp

@@ -81,11 +81,13 @@ def test_spmm_exact_on_integers_and_strided_tensors(S):
         S.spdp_free(h)
 
 
-@pytest.mark.parametrize("R,K,N", [(80, 200, 1), (80, 200, 256), (80, 72, 300), (40, 136, 600), (30, 264, 700), (3, 520, 1100)])
+@pytest.mark.parametrize("R,K,N", [(80, 200, 1), (80, 200, 256), (80, 72, 300), (40, 136, 600), (30, 264, 700), (3, 520, 1100),
+                                   (76, 264, 100), (150, 520, 300), (75, 2048, 700)])
 def test_spmm_both_kernels(S, R, K, N):
     """The launch chooses between a CTA per row tile (256 tokens) and a CTA pair per row tile (512 tokens) by the
     rounds of CTAs each needs: many row tiles with few tokens take the first, the rest the second.  These shapes
-    reach both, with one and with several token blocks, ragged in M, K and N."""
+    reach both, with one and with several token blocks, ragged in M, K and N.  The last three leave a last round of
+    two CTA pairs on a 148-SM GPU: those tiles are cut along K and their slices added by a second kernel."""
     rw, rx = WL._rngs(100 + R)
     M = 256 * R - 37
     W = WL.prune_global_magnitude(WL.normal_weights(rw, M, K), 0.5).astype(np.float16)
@@ -93,8 +95,10 @@ def test_spmm_both_kernels(S, R, K, N):
     Y_ref, S_ref = O.spmm_ref(W, X)
     h = S.spdp_pack_tiled_cbc(dev(W))
     try:
-        check(run(S, h, X, M), Y_ref, S_ref)
+        y = run(S, h, X, M)
+        check(y, Y_ref, S_ref)
         check(run(S, h, X, M, torch.float16), Y_ref, S_ref)
+        assert np.array_equal(y, run(S, h, X, M))                       # the same bits from call to call
     finally:
         S.spdp_free(h)
 

@@ -19,7 +19,7 @@
 //     block's tcgen05.mma (K = 16 each) and commits them to the stage's barrier.
 //   * 16 decode warps: warp w decodes columns w, w+16, w+32, w+48 of the block into the operand tile
 //     and arrives on the stage's barriers.  They issue no copies and meet no CTA-wide barrier in the loop.
-// Every wait is bounded; no copy is multicast.
+// Every wait is bounded; every copy writes only the shared memory of the CTA that issued it.
 //
 // Two kernels share this structure:
 //   one::spmm_kernel   one CTA = one row tile (256 rows = two M = 128 accumulators) x 256 tokens.

@@ -39,9 +39,10 @@ using namespace dev;
 constexpr int kWarps = SPDP_Q4_WARPS;         // warps per CTA; every warp fetches and decodes its own column tiles
 constexpr int kDepth = SPDP_Q4_DEPTH;         // groups a warp keeps in flight
 constexpr int kGroup = 4;                  // active column tiles per group (one fetch / decode unit of a warp)
-constexpr int kSlotBytes = kTileM / 2 + 16;  // a column tile's codes (at most 256 nibbles) + 16 bytes: the decode reads
-                                             // two 32-bit words from the span's first, and the four tiles of a group
-                                             // start 4 banks apart
+constexpr int kSlotPad = 16;                 // bytes in front of a slot's codes: the decode reads the two 32-bit words that
+                                             // END at a lane's last code, the first of which may lie before the codes
+constexpr int kSlotBytes = kSlotPad + kTileM / 2;   // + a column tile's codes (at most 256 nibbles); the four tiles of a
+                                                    // group start 4 banks apart
 constexpr int kStageBytes = kGroup * kSlotBytes;
 constexpr int kThreads = kWarps * 32;
 constexpr int kChunkCols = SPDP_Q4_CHUNK_COLS; // columns handled between two pipeline drains
@@ -103,12 +104,15 @@ static_assert(sizeof(Smem) <= (227 * 1024) / kCtasPerSm - 1024 * (kCtasPerSm - 1
 static_assert(kRecPad <= kThreads, "one thread per trailing null record");
 static_assert(kWarps >= 16, "two groups of 256 threads finish two row tiles side by side");
 
-// The walk over a lane's 8 rows (Sec. 4.2.1 with 4-bit codes): a set bit takes the next nibble of `span`;
-// (code | 0x4B000000) is 2^23 + code as a float, so one subtraction turns the code into code - 8 without a
-// conversion; acc[row] += (code - 8) * (scale * x).  Five instructions per row, the last two predicated.
+// The walk over a lane's 8 rows (Sec. 4.2.1 with 4-bit codes), from the last row to the first: `span` holds the
+// lane's codes with the LAST one in the top nibble; a set bit takes the top nibble and shifts the span left.
+// mad.hi(span, 16, 2^23-as-float bits) = (span >> 28) | 0x4B000000 = 2^23 + code as a float, so one subtraction
+// turns the code into code - 8 without a conversion; acc[row] += (code - 8) * (scale * x).  Five instructions per
+// row, the last two predicated; only the bit test uses the integer pipe (the multiply-high, the subtraction, the
+// FMA and the shift-as-multiply go to the FMA pipe).
 #define SPDP_Q4_ROW(K)                                              \
     " lop3.or.b32 t|p, %9, " #K ", 0, 0xC0, 0;\n"                  \
-    " lop3.b32 c, %8, 15, 0x4B000000, 0xEA;\n"                     \
+    " mad.hi.u32 c, %8, 16, 0x4B000000;\n"                         \
     " add.f32 w, c, 0fCB000008;\n"
 __device__ __forceinline__ void walk_codes(unsigned bits, unsigned span, float sx, float (&acc)[8]) {
     asm volatile(
@@ -116,14 +120,14 @@ __device__ __forceinline__ void walk_codes(unsigned bits, unsigned span, float s
         " .reg .pred p;\n"
         " .reg .b32 t, c;\n"
         " .reg .f32 w;\n"
-        SPDP_Q4_ROW(1)   " @p fma.rn.f32 %0, w, %10, %0;\n @p shr.b32 %8, %8, 4;\n"
-        SPDP_Q4_ROW(2)   " @p fma.rn.f32 %1, w, %10, %1;\n @p shr.b32 %8, %8, 4;\n"
-        SPDP_Q4_ROW(4)   " @p fma.rn.f32 %2, w, %10, %2;\n @p shr.b32 %8, %8, 4;\n"
-        SPDP_Q4_ROW(8)   " @p fma.rn.f32 %3, w, %10, %3;\n @p shr.b32 %8, %8, 4;\n"
-        SPDP_Q4_ROW(16)  " @p fma.rn.f32 %4, w, %10, %4;\n @p shr.b32 %8, %8, 4;\n"
-        SPDP_Q4_ROW(32)  " @p fma.rn.f32 %5, w, %10, %5;\n @p shr.b32 %8, %8, 4;\n"
-        SPDP_Q4_ROW(64)  " @p fma.rn.f32 %6, w, %10, %6;\n @p shr.b32 %8, %8, 4;\n"
-        SPDP_Q4_ROW(128) " @p fma.rn.f32 %7, w, %10, %7;\n"
+        SPDP_Q4_ROW(128) " @p fma.rn.f32 %7, w, %10, %7;\n @p mul.lo.u32 %8, %8, 16;\n"
+        SPDP_Q4_ROW(64)  " @p fma.rn.f32 %6, w, %10, %6;\n @p mul.lo.u32 %8, %8, 16;\n"
+        SPDP_Q4_ROW(32)  " @p fma.rn.f32 %5, w, %10, %5;\n @p mul.lo.u32 %8, %8, 16;\n"
+        SPDP_Q4_ROW(16)  " @p fma.rn.f32 %4, w, %10, %4;\n @p mul.lo.u32 %8, %8, 16;\n"
+        SPDP_Q4_ROW(8)   " @p fma.rn.f32 %3, w, %10, %3;\n @p mul.lo.u32 %8, %8, 16;\n"
+        SPDP_Q4_ROW(4)   " @p fma.rn.f32 %2, w, %10, %2;\n @p mul.lo.u32 %8, %8, 16;\n"
+        SPDP_Q4_ROW(2)   " @p fma.rn.f32 %1, w, %10, %1;\n @p mul.lo.u32 %8, %8, 16;\n"
+        SPDP_Q4_ROW(1)   " @p fma.rn.f32 %0, w, %10, %0;\n"
         "}"
         : "+f"(acc[0]), "+f"(acc[1]), "+f"(acc[2]), "+f"(acc[3]), "+f"(acc[4]), "+f"(acc[5]), "+f"(acc[6]), "+f"(acc[7]),
           "+r"(span)
@@ -191,7 +195,7 @@ spmspv_q4_kernel(const Params p) {
     const int tpos = lgrp * 8 + lane7;                                  // where (tile lgrp, word lane7) sits
     const unsigned bsh = pinned(8u * (lane & 3));
     const unsigned bbelow = pinned((1u << (8 * (lane & 3))) - 1u);      // the bits of my word below my byte
-    const uint32_t val_dst = pinned(smem_u32(&sm.ring[warp][0][lgrp * kSlotBytes + 16 * lane7]));
+    const uint32_t val_dst = pinned(smem_u32(&sm.ring[warp][0][lgrp * kSlotBytes + kSlotPad + 16 * lane7]));
     const uint32_t bm_own = pinned(smem_u32(&sm.tab[warp].bm[0][tpos]));
     const uint32_t bm_dec = pinned(smem_u32(&sm.tab[warp].bm[0][lane >> 2]));
     constexpr int kVoFromBm = kDepth * 128;             // vo[d][i] sits this many bytes behind bm[d][i]
@@ -433,9 +437,11 @@ spmspv_q4_kernel(const Params p) {
                 const unsigned W = lds_u32(bmd + 32 * it);
                 const unsigned rank = lds_u32(bmd + 32 * it + kVoFromBm) + __popc(W & bbelow);   // codes before my byte
                 const unsigned bits = (W >> bsh) & 0xFFu;
-                // my codes: at most 8 nibbles from nibble `rank` on, inside two consecutive 32-bit words of the slot
-                const uint32_t cw = ring_warp + dv + it * kSlotBytes + 4u * (rank >> 3);
-                const unsigned span = __funnelshift_r(lds_u32(cw), lds_u32(cw + 4), 4u * (rank & 7u));
+                // my codes: the at most 8 nibbles that end before nibble `rend`, inside the two consecutive 32-bit words
+                // that end with the word of nibble `rend` (the word before the codes is padding); last code on top
+                const unsigned rend = rank + __popc(bits);
+                const uint32_t cw = ring_warp + dv + it * kSlotBytes + (kSlotPad - 4) + 4u * (rend >> 3);
+                const unsigned span = __funnelshift_r(lds_u32(cw), lds_u32(cw + 4), 4u * (rend & 7u));
                 walk_codes(bits, span, sx[it], acc);
             }
             __syncwarp();                  // everyone is done with this ring position

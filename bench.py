@@ -392,6 +392,38 @@ def run_prefill(args):
     spdp.spdp_free(h)
 
 
+def graph_replay_stats(step, copies):
+    """The calls `step(i)` replayed from a CUDA graph (>= 100 calls, whole rotations over the packed copies), so that
+    the launch overhead is out of the picture: per-call time over 10 replays."""
+    import torch
+    calls = copies * max(1, -(-100 // copies))
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        for i in range(copies):
+            step(i)
+        side.synchronize()
+        with torch.cuda.graph(g, stream=side):
+            for i in range(calls):
+                step(i)
+        for _ in range(10):
+            g.replay()
+        side.synchronize()
+        per_call = []
+        for _ in range(10):
+            g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            g0.record(side)
+            g.replay()
+            g1.record(side)
+            side.synchronize()
+            per_call.append(g0.elapsed_time(g1) / calls * 1e3)
+    torch.cuda.current_stream().wait_stream(side)
+    del g
+    return {"calls_per_graph": calls, "replays": 10, "us_per_call_min": min(per_call),
+            "us_per_call_median": float(np.median(per_call)), "us_per_call_max": max(per_call)}
+
+
 def run_q4(args):
     """--q4: the decode call on the 4-bit Values variant of the same layer (Sec. 5.1 / Sec. 6).  A side
     measurement: the byte model shrinks to half a byte per stored weight plus one fp16 scale per column tile."""
@@ -422,6 +454,10 @@ def run_q4(args):
     e1.record()
     torch.cuda.synchronize()
     us = e0.elapsed_time(e1) / args.steps * 1e3
+    graph_stats = None
+    if not args.no_graph:
+        graph_stats = graph_replay_stats(
+            lambda i: spdp.spdp_spmspv(handles[i % copies], xs[i % copies], w.rule, w.thr, ys[i % copies]), copies)
     assert all(spdp.spdp_last_device_status(h) == 0 for h in handles)
     # parity on the rows of three row tiles, against the oracle's product on the dequantised weights
     yh = ys[0].float().cpu().numpy().astype(np.float64)
@@ -441,7 +477,7 @@ def run_q4(args):
         "config": {"workload": w.name, "storage": "4-bit codes + fp16 scale per column tile", "active_bytes_per_call": int(B_active),
                    "packed_bytes": int(info.packed_bytes), "copies": copies,
                    "l2": "inputs larger than L2: rotating packed copies"},
-        "gpu_launches": args.steps,
+        "gpu_launches": args.steps, "graph": graph_stats,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_kind": f"of {peak_kind}", "traffic": None, "kernel": "spmspv_q4_kernel",
                      "algorithmic_bytes": int(B_active)},
@@ -738,32 +774,7 @@ def main():
     # ---- the same calls replayed from a CUDA graph (launch overhead out of the picture) ----
     graph_stats = None
     if not args.no_graph:
-        calls = copies * max(1, -(-100 // copies))              # >= 100 calls, whole rotations
-        side = torch.cuda.Stream()
-        side.wait_stream(torch.cuda.current_stream())
-        g = torch.cuda.CUDAGraph()
-        with torch.cuda.stream(side):
-            for i in range(copies):
-                step(i)
-            side.synchronize()
-            with torch.cuda.graph(g, stream=side):
-                for i in range(calls):
-                    step(i)
-            for _ in range(10):
-                g.replay()
-            side.synchronize()
-            per_call = []
-            for _ in range(10):
-                g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                g0.record(side)
-                g.replay()
-                g1.record(side)
-                side.synchronize()
-                per_call.append(g0.elapsed_time(g1) / calls * 1e3)
-        torch.cuda.current_stream().wait_stream(side)
-        graph_stats = {"calls_per_graph": calls, "replays": 10, "us_per_call_min": min(per_call),
-                       "us_per_call_median": float(np.median(per_call)), "us_per_call_max": max(per_call)}
-        del g
+        graph_stats = graph_replay_stats(step, copies)
 
     # ---- end to end through the host-vector entry point ----------------------------------
     xh = torch.from_numpy(w.x.copy()).pin_memory()
